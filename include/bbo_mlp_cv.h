@@ -1,0 +1,140 @@
+/* bbo_mlp_cv.h -- C ABI of the fused MLP-Adam cross-validation library (CUDA, sm_100a).
+ *
+ * The library is the `evaluate(params_list) -> scores` call of the suggest-observe loop
+ * (paper, Algorithm 1): for every suggested hyperparameter configuration it returns "the
+ * cross validation score of a machine learning model on a dataset with a loss function"
+ * (paper, sec. 2) for the model the paper's Table 1 calls MLP-adam, with the metrics acc
+ * and mse of the same table, five folds in the paper's runs (sec. 6.3: 2.7 M trainings for
+ * 541,440 evaluations).  Function evaluation is what the paper moves to the GPU because it
+ * dominates run time (sec. 1, sec. 5, sec. 6.3).
+ *
+ * Model and training rule (the paper names the model, not its formulas; these are the
+ * readings this library fixes): one hidden ReLU layer of width `hidden`; softmax
+ * cross-entropy averaged over the minibatch (classification) or half the mean squared error
+ * (regression); L2 penalty alpha/(2*batch) on both weight matrices; Adam with step size
+ * lr*sqrt(1-beta2^t)/(1-beta1^t) and update m/(sqrt(v)+eps); Glorot-uniform initial
+ * weights and biases; shuffled, non-stratified k-fold split shared by all configurations;
+ * a fresh minibatch permutation every epoch, last short batch kept.  All random choices come
+ * from Philox-4x32-10 keyed by `seed` and indexed by (configuration index, fold, epoch or
+ * layer, element), so a score depends only on its own configuration, its index in the list
+ * and the seed -- never on the other entries, the grid or the scheduling.
+ *
+ * No C++ types, no exceptions and no printing cross this boundary.  Every function returns
+ * 0 on success or a negative bbo_status.  All floating point is IEEE binary32 unless noted.
+ */
+#ifndef BBO_MLP_CV_H_
+#define BBO_MLP_CV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bbo_mlp_cv bbo_mlp_cv; /* opaque handle */
+
+/* One suggested configuration (an element of Algorithm 1's params_list).  POD, 32 bytes. */
+typedef struct {
+  int32_t hidden;     /* H >= 1, at most the cap reported by bbo_mlp_cv_query_caps        */
+  int32_t batch_size; /* B >= 1; the effective size is min(B, training rows of the fold)   */
+  int32_t epochs;     /* E in [0, 2^28); 0 scores the initial weights                      */
+  float alpha;        /* L2 strength >= 0                                                   */
+  float lr;           /* Adam learning rate >= 0                                            */
+  float beta1, beta2; /* in [0, 1)                                                          */
+  float eps;          /* > 0                                                                */
+} bbo_mlp_config;
+
+typedef enum { BBO_TASK_CLASSIFICATION = 0, BBO_TASK_REGRESSION = 1 } bbo_task;
+
+typedef enum {
+  BBO_OK = 0,
+  BBO_ERR_INVALID_ARG = -1, /* NULL pointer, bad size, hyperparameter or label out of range */
+  BBO_ERR_UNSUPPORTED = -2, /* shape above the kernel caps, or not an sm_100 device         */
+  BBO_ERR_CUDA = -3,        /* a CUDA runtime call failed (see bbo_mlp_cv_last_cuda_error)  */
+  BBO_ERR_TIMEOUT = -4,     /* a bounded device-side wait gave up                           */
+  BBO_ERR_OOM = -5          /* scratch allocation failed                                    */
+} bbo_status;
+
+/* Create-time options; a zeroed struct selects the defaults. */
+typedef struct {
+  int32_t device;      /* CUDA ordinal; -1 = the calling thread's current device            */
+  void* stream;        /* cudaStream_t borrowed from the caller; NULL = the default stream  */
+  int32_t n_classes;   /* classification: 0 = 1 + max(y) found on the device                */
+  int32_t trace_steps; /* >0: record the minibatch training loss of the first N optimizer
+                          steps of every fit (debug / parity; slows the kernel)             */
+  int32_t keep_theta;  /* 1: keep the final parameters of the LAST fit of the list, i.e.
+                          (configuration n_configs-1, fold n_folds-1), for
+                          bbo_mlp_cv_debug_theta                                            */
+  int32_t reserved[3];
+} bbo_mlp_cv_options;
+
+/* Creates a handle bound to one device and one stream.  `opt` may be NULL (defaults).
+ * The handle owns its scratch buffers (grown on demand, freed by destroy).               */
+int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out);
+
+/* scores = evaluate(params_list) (paper, Algorithm 1; sec. 2).
+ *   X          DEVICE, row-major [n*d] float, 4-byte aligned; read only
+ *   y          DEVICE [n] float: class ids 0..C-1 stored exactly, or regression targets
+ *   n, d       rows and features; task  a bbo_task; n_folds  2 <= K <= n
+ *   configs    HOST [n_configs]; copied during the call
+ *   seed       keys the fold split, every initialisation and every minibatch order
+ *   out_scores DEVICE [n_configs] float: mean over folds (ascending fold, float sum, then
+ *              one division) of held-out accuracy, or of minus the held-out mean squared
+ *              error (higher is better; a NaN error maps to -inf)
+ * Work is enqueued on the handle's stream, which is synchronised before returning, so the
+ * status reflects the device's and out_scores is ready.  The caller keeps ownership of all
+ * four buffers; none is retained.  On error out_scores is unspecified.  One call at a time
+ * per handle; distinct handles are independent.                                           */
+int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d,
+                    int32_t task, int32_t n_folds, const bbo_mlp_config* configs,
+                    int32_t n_configs, uint64_t seed, float* out_scores);
+
+/* As bbo_mlp_cv_eval, with X, y and out_scores in HOST memory: copies them to device
+ * scratch owned by the handle, evaluates, copies the scores back.                         */
+int bbo_mlp_cv_eval_host(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d,
+                         int32_t task, int32_t n_folds, const bbo_mlp_config* configs,
+                         int32_t n_configs, uint64_t seed, float* out_scores);
+
+int bbo_mlp_cv_destroy(bbo_mlp_cv* h);
+
+/* Results of the last eval kept by the handle (HOST output buffers).
+ *   fold_scores: [n_configs*n_folds], configuration-major
+ *   loss_trace:  [n_configs*n_folds*trace_steps], NaN where a fit had fewer steps
+ *   theta:       W1[d][H] row-major, b1[H], W2[H][C] row-major, b2[C] of the kept fit;
+ *                `count` must equal that parameter count                                  */
+int bbo_mlp_cv_fold_scores(bbo_mlp_cv* h, float* host_out, int64_t count);
+int bbo_mlp_cv_loss_trace(bbo_mlp_cv* h, float* host_out, int64_t count);
+int bbo_mlp_cv_debug_theta(bbo_mlp_cv* h, float* host_out, int64_t count);
+
+/* Runs the DEVICE index code and copies the result back (parity of the fold split and the
+ * minibatch order).  host_fold_of_row[n]: fold in which each row is held out.
+ * host_order[n - size of that fold]: dataset row visited i-th in `epoch` of fit
+ * (config, fold); minibatch s of size B is host_order[s*B .. s*B+B).  Either may be NULL. */
+int bbo_mlp_cv_debug_indices(bbo_mlp_cv* h, int64_t n, int32_t n_folds, uint64_t seed,
+                             int32_t config, int32_t fold, int32_t epoch,
+                             int32_t* host_fold_of_row, int32_t* host_order);
+
+/* Device-side Philox block and the float exponential used by the softmax, for bit-exact
+ * comparison with another implementation.  counters: HOST [count*5] words
+ * (stream, a, b, c, blk); out: HOST [count*4].  x, out: HOST [count].                     */
+int bbo_mlp_cv_debug_rng(bbo_mlp_cv* h, uint64_t seed, const uint32_t* counters, int64_t count,
+                         uint32_t* out);
+int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* out);
+
+/* Largest shapes one call accepts on this device: rows, features, hidden width for the
+ * given (d, n_classes) pair, and classes.  Any output pointer may be NULL.               */
+int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* max_n,
+                          int32_t* max_d, int32_t* max_hidden, int32_t* max_classes);
+
+/* Device time of the last eval's kernels (fold split .. fold mean) in milliseconds, and the
+ * number of kernels it launched.  Either pointer may be NULL.                             */
+int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* kernel_ms, int32_t* n_launches);
+
+const char* bbo_mlp_cv_strerror(int code);
+/* Text of the last CUDA error seen by this handle ("" if none).  Valid until the next call. */
+const char* bbo_mlp_cv_last_cuda_error(bbo_mlp_cv* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BBO_MLP_CV_H_ */

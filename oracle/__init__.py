@@ -58,6 +58,10 @@ def lib():
         L.oracle_epoch_order.restype = ctypes.c_int
         L.oracle_expf.argtypes = [ctypes.c_float]
         L.oracle_expf.restype = ctypes.c_float
+        L.oracle_expf_array.argtypes = [vp, i64, vp]
+        L.oracle_expf_array.restype = None
+        L.oracle_rng_blocks.argtypes = [u64, vp, i64, vp]
+        L.oracle_rng_blocks.restype = None
         L.oracle_param_count.argtypes = [i32, i32, i32]
         L.oracle_param_count.restype = i64
         L.oracle_init_params.argtypes = [i32, i32, i32, u64, i32, i32, vp]
@@ -120,6 +124,21 @@ def epoch_order(n, K, seed, config, fold, epoch):
 
 def expf(x):
     return float(lib().oracle_expf(float(x)))
+
+
+def expf_array(x):
+    x = np.ascontiguousarray(x, np.float32)
+    out = np.empty_like(x)
+    lib().oracle_expf_array(_p(x), x.size, _p(out))
+    return out
+
+
+def rng_blocks(seed, counters):
+    """counters [count, 5] = (stream, a, b, c, blk) -> words [count, 4]."""
+    counters = np.ascontiguousarray(counters, np.uint32).reshape(-1, 5)
+    out = np.empty((counters.shape[0], 4), np.uint32)
+    lib().oracle_rng_blocks(seed, _p(counters), counters.shape[0], _p(out))
+    return out
 
 
 def param_count(d, H, C):

@@ -422,6 +422,17 @@ int oracle_epoch_order(int64_t n, int32_t K, uint64_t seed, int32_t config, int3
 
 float oracle_expf(float x) { return spec_expf(x); }
 
+void oracle_expf_array(const float* x, int64_t count, float* out) {
+  for (int64_t i = 0; i < count; ++i) out[i] = spec_expf(x[i]);
+}
+
+// counters[count][5] = (stream, a, b, c, blk) -> out[count][4]
+void oracle_rng_blocks(uint64_t seed, const uint32_t* counters, int64_t count, uint32_t* out) {
+  for (int64_t i = 0; i < count; ++i)
+    philox_block(seed, counters[5 * i], counters[5 * i + 1], counters[5 * i + 2], counters[5 * i + 3],
+                 counters[5 * i + 4], out + 4 * i);
+}
+
 int64_t oracle_param_count(int32_t d, int32_t H, int32_t C) { return Shape{d, H, C}.P(); }
 
 void oracle_init_params(int32_t d, int32_t H, int32_t C, uint64_t seed, int32_t config, int32_t fold,

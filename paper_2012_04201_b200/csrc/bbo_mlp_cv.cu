@@ -1,0 +1,506 @@
+// Host side of the C ABI declared in include/bbo_mlp_cv.h: argument checks, scratch
+// management, the launch sequence (label scan, row padding, fold permutation, the fit
+// kernel, fold mean) and the debug exports.  scores = evaluate(params_list) of the paper's
+// Algorithm 1, with the cross-validation score of sec. 2 as the evaluated function.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/bbo_mlp_cv.h"
+#include "fit_kernel.cuh"
+
+static_assert(sizeof(bbo_mlp_config) == 32, "bbo_mlp_config must be 32 bytes");
+static_assert(sizeof(bbo::Config) == sizeof(bbo_mlp_config), "device mirror of bbo_mlp_config");
+
+namespace {
+
+constexpr int kMaxClasses = 16;
+constexpr int kMaxThreads = 512;
+constexpr int kMaxRows = 16384;  // fold permutation sorts in one CTA's shared memory
+
+template <typename T>
+struct DevBuf {
+  T* p = nullptr;
+  size_t cap = 0;
+  cudaError_t reserve(size_t n) {
+    if (n <= cap) return cudaSuccess;
+    if (p) cudaFree(p);
+    p = nullptr;
+    cap = 0;
+    cudaError_t e = cudaMalloc(&p, n * sizeof(T));
+    if (e == cudaSuccess) cap = n;
+    return e;
+  }
+  void release() {
+    if (p) cudaFree(p);
+    p = nullptr;
+    cap = 0;
+  }
+};
+
+}  // namespace
+
+struct bbo_mlp_cv {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  bbo_mlp_cv_options opt{};
+  int sm_count = 0;
+  int smem_optin = 0;
+  std::string cuda_error;
+  // scratch
+  DevBuf<bbo::Config> configs;
+  DevBuf<int2> fits;
+  DevBuf<float> fold_scores, trace, theta, xpad, hx, hy, hscores, dbg_f;
+  DevBuf<int32_t> pi, misc, dbg_i;
+  DevBuf<uint32_t> dbg_u;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  // last eval
+  int64_t last_fold_count = 0, last_trace_count = 0, last_theta_count = 0;
+  float last_ms = 0.f;
+  int last_launches = 0;
+};
+
+namespace {
+
+int cuda_fail(bbo_mlp_cv* h, cudaError_t e, const char* what) {
+  h->cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return e == cudaErrorMemoryAllocation ? BBO_ERR_OOM : BBO_ERR_CUDA;
+}
+
+#define BBO_CUDA(h, call)                                       \
+  do {                                                          \
+    cudaError_t e_ = (call);                                    \
+    if (e_ != cudaSuccess) return cuda_fail((h), e_, #call);    \
+  } while (0)
+
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) {
+    cudaGetDevice(&prev);
+    if (prev != dev) cudaSetDevice(dev);
+    else prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+bool is_device_ptr(const void* p, int device) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return (at.type == cudaMemoryTypeDevice && at.device == device) || at.type == cudaMemoryTypeManaged;
+}
+
+struct Plan {
+  int C, CS, dp, TB, NT, order_bytes, loss_cap, n_sort;
+  size_t smem;
+};
+
+// Threads needed by a fit of width H: one per gradient tile (4 rows x 8 columns of W1) and
+// one per hidden unit.
+int threads_for(int dp, int H) {
+  const int Hs = bbo::round_up(H, 8);
+  const int tiles = (dp / 4) * (Hs / 8);
+  return bbo::round_up(std::max(std::max(tiles, Hs), 64), 32);
+}
+
+size_t smem_for(int d, int dp, int H, int CS, int TB, int order_bytes, int loss_cap, int n_sort) {
+  bbo::Layout L(d, H, CS);
+  return 3u * (size_t)L.PS * 4u + bbo::scratch_bytes(L.Hs, dp, CS, TB, order_bytes, loss_cap, n_sort);
+}
+
+// Largest sub-tile height (64, 32, ... 4) for which the widest fit fits in shared memory.
+int plan_launch(const bbo_mlp_cv* h, int n, int d, int C, int K, int maxH, int maxB, bool tracing, Plan* out) {
+  Plan p{};
+  p.C = C;
+  p.CS = bbo::round_up(C, 4);
+  p.dp = bbo::round_up(d, 4);
+  const int n_tr_max = n - n / K;
+  p.order_bytes = bbo::round_up(2 * n_tr_max, 16);
+  p.loss_cap = tracing ? std::min(maxB, n_tr_max) : 0;
+  p.n_sort = n_tr_max;
+  p.NT = threads_for(p.dp, maxH);
+  if (p.NT > kMaxThreads) return BBO_ERR_UNSUPPORTED;
+  const size_t budget = (size_t)h->smem_optin - 256;  // static block scalars
+  for (int TB = 32; TB >= 4; TB >>= 1) {
+    const size_t need = smem_for(d, p.dp, maxH, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort);
+    if (need <= budget) {
+      p.TB = TB;
+      p.smem = need;
+      *out = p;
+      return BBO_OK;
+    }
+  }
+  return BBO_ERR_UNSUPPORTED;
+}
+
+template <typename Kern>
+cudaError_t launch_kernel(Kern kern, const bbo::FitArgs& a, int n_sm, int NT, size_t smem, cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NT, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  const int grid = std::min(a.n_fits, n_sm * per_sm);  // persistent CTAs, all resident
+  kern<<<grid, NT, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
+template <int CT>
+cudaError_t launch_fit(const bbo::FitArgs& a, int n_sm, int NT, size_t smem, cudaStream_t s) {
+  if (NT <= 256) return launch_kernel(bbo::mlp_cv_fit_kernel<CT, 256>, a, n_sm, NT, smem, s);
+  return launch_kernel(bbo::mlp_cv_fit_kernel<CT, 512>, a, n_sm, NT, smem, s);
+}
+
+cudaError_t launch_fit_any(int C, const bbo::FitArgs& a, int n_sm, int NT, size_t smem, cudaStream_t s) {
+  switch (C) {
+    case 1: return launch_fit<1>(a, n_sm, NT, smem, s);
+    case 2: return launch_fit<2>(a, n_sm, NT, smem, s);
+    case 3: return launch_fit<3>(a, n_sm, NT, smem, s);
+    case 10: return launch_fit<10>(a, n_sm, NT, smem, s);
+    default: return C <= 4 ? launch_fit<4>(a, n_sm, NT, smem, s) : launch_fit<kMaxClasses>(a, n_sm, NT, smem, s);
+  }
+}
+
+cudaError_t launch_fold_permutation(int n, uint64_t seed, int32_t* pi, cudaStream_t s) {
+  const size_t bytes = 8u * (size_t)bbo::next_pow2(n);
+  cudaError_t e = cudaFuncSetAttribute(bbo::fold_permutation_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e != cudaSuccess) return e;
+  bbo::fold_permutation_kernel<<<1, 1024, bytes, s>>>(n, seed, pi);
+  return cudaGetLastError();
+}
+
+int check_configs(const bbo_mlp_config* cfg, int n_configs, int* maxH, int* maxB) {
+  *maxH = 1;
+  *maxB = 1;
+  for (int c = 0; c < n_configs; ++c) {
+    const bbo_mlp_config& q = cfg[c];
+    if (q.hidden < 1 || q.batch_size < 1 || q.epochs < 0 || q.epochs >= (1 << 28)) return BBO_ERR_INVALID_ARG;
+    if (!(q.alpha >= 0.f) || !std::isfinite(q.alpha) || !(q.lr >= 0.f) || !std::isfinite(q.lr)) return BBO_ERR_INVALID_ARG;
+    if (!(q.beta1 >= 0.f && q.beta1 < 1.f) || !(q.beta2 >= 0.f && q.beta2 < 1.f)) return BBO_ERR_INVALID_ARG;
+    if (!(q.eps > 0.f) || !std::isfinite(q.eps)) return BBO_ERR_INVALID_ARG;
+    *maxH = std::max(*maxH, q.hidden);
+    *maxB = std::max(*maxB, q.batch_size);
+  }
+  return BBO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out) {
+  if (!out) return BBO_ERR_INVALID_ARG;
+  *out = nullptr;
+  bbo_mlp_cv_options o{};
+  if (opt) o = *opt;
+  else o.device = -1;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0) {
+    cudaGetLastError();
+    return BBO_ERR_CUDA;
+  }
+  int dev = o.device;
+  if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return BBO_ERR_CUDA;
+  if (dev >= count || o.n_classes < 0 || o.n_classes > kMaxClasses || o.trace_steps < 0) return BBO_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return BBO_ERR_CUDA;
+  if (prop.major != 10) return BBO_ERR_UNSUPPORTED;  // the kernels are built for sm_100a only
+  bbo_mlp_cv* h = new (std::nothrow) bbo_mlp_cv();
+  if (!h) return BBO_ERR_OOM;
+  h->device = dev;
+  h->stream = static_cast<cudaStream_t>(o.stream);
+  h->opt = o;
+  h->sm_count = prop.multiProcessorCount;
+  h->smem_optin = (int)prop.sharedMemPerBlockOptin;
+  DeviceGuard g(dev);
+  if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess) {
+    delete h;
+    return BBO_ERR_CUDA;
+  }
+  *out = h;
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_destroy(bbo_mlp_cv* h) {
+  if (!h) return BBO_ERR_INVALID_ARG;
+  DeviceGuard g(h->device);
+  cudaStreamSynchronize(h->stream);
+  h->configs.release(); h->fits.release(); h->fold_scores.release(); h->trace.release();
+  h->theta.release(); h->xpad.release(); h->hx.release(); h->hy.release(); h->hscores.release();
+  h->dbg_f.release(); h->pi.release(); h->misc.release(); h->dbg_i.release(); h->dbg_u.release();
+  if (h->ev0) cudaEventDestroy(h->ev0);
+  if (h->ev1) cudaEventDestroy(h->ev1);
+  delete h;
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, int32_t d, int32_t task,
+                    int32_t K, const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed,
+                    float* out_scores) {
+  if (!h || !X || !y || !configs || !out_scores) return BBO_ERR_INVALID_ARG;
+  if (n64 < 2 || d < 1 || K < 2 || K > n64 || n_configs < 1) return BBO_ERR_INVALID_ARG;
+  if (task != BBO_TASK_CLASSIFICATION && task != BBO_TASK_REGRESSION) return BBO_ERR_INVALID_ARG;
+  if (n64 > kMaxRows || (int64_t)n_configs * K > (1 << 30) || n_configs >= (1 << 28)) return BBO_ERR_UNSUPPORTED;
+  int maxH, maxB;
+  int rc = check_configs(configs, n_configs, &maxH, &maxB);
+  if (rc != BBO_OK) return rc;
+  DeviceGuard g(h->device);
+  if (!is_device_ptr(X, h->device) || !is_device_ptr(y, h->device) || !is_device_ptr(out_scores, h->device))
+    return BBO_ERR_INVALID_ARG;
+  const int n = (int)n64;
+  cudaStream_t s = h->stream;
+  h->cuda_error.clear();
+  h->last_fold_count = h->last_trace_count = h->last_theta_count = 0;
+
+  // misc[0] = work counter, misc[1] = max label, misc[2] = bad-label flag
+  BBO_CUDA(h, h->misc.reserve(4));
+  BBO_CUDA(h, cudaMemsetAsync(h->misc.p, 0, 4 * sizeof(int32_t), s));
+  int launches = 0;
+  int C = 1;
+  if (task == BBO_TASK_CLASSIFICATION) {
+    bbo::label_scan_kernel<<<std::min(64, (n + 255) / 256), 256, 0, s>>>(y, n, h->misc.p + 1);
+    BBO_CUDA(h, cudaGetLastError());
+    ++launches;
+    int32_t info[2];
+    BBO_CUDA(h, cudaMemcpyAsync(info, h->misc.p + 1, sizeof(info), cudaMemcpyDeviceToHost, s));
+    BBO_CUDA(h, cudaStreamSynchronize(s));
+    if (info[1] != 0) return BBO_ERR_INVALID_ARG;
+    C = info[0] + 1;
+    if (h->opt.n_classes > 0) {
+      if (C > h->opt.n_classes) return BBO_ERR_INVALID_ARG;
+      C = h->opt.n_classes;
+    }
+    if (C > kMaxClasses) return BBO_ERR_UNSUPPORTED;
+  }
+
+  Plan plan;
+  const bool tracing = h->opt.trace_steps > 0;
+  rc = plan_launch(h, n, d, C, K, maxH, maxB, tracing, &plan);
+  if (rc != BBO_OK) return rc;
+
+  const int n_fits = n_configs * K;
+  // fit list, costliest first: E * n_train * (4dH + 6HC) + steps * 14 P
+  std::vector<int2> fits((size_t)n_fits);
+  {
+    std::vector<std::pair<double, int>> cost((size_t)n_fits);
+    for (int c = 0; c < n_configs; ++c) {
+      const bbo_mlp_config& q = configs[c];
+      for (int f = 0; f < K; ++f) {
+        int vb, vs;
+        bbo::fold_segment(n, K, f, &vb, &vs);
+        const double n_tr = n - vs, B = std::min<double>(q.batch_size, n_tr);
+        const double P = (double)d * q.hidden + q.hidden + (double)q.hidden * C + C;
+        const double steps = (double)q.epochs * std::ceil(n_tr / B);
+        cost[(size_t)c * K + f] = {(double)q.epochs * n_tr * (4.0 * d * q.hidden + 6.0 * q.hidden * C) + steps * 14.0 * P,
+                                   c * K + f};
+      }
+    }
+    std::stable_sort(cost.begin(), cost.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
+    for (int i = 0; i < n_fits; ++i) fits[i] = make_int2(cost[i].second / K, cost[i].second % K);
+  }
+
+  BBO_CUDA(h, h->configs.reserve(n_configs));
+  BBO_CUDA(h, h->fits.reserve(n_fits));
+  BBO_CUDA(h, h->fold_scores.reserve(n_fits));
+  BBO_CUDA(h, h->pi.reserve(n));
+  BBO_CUDA(h, cudaMemcpyAsync(h->configs.p, configs, sizeof(bbo_mlp_config) * (size_t)n_configs, cudaMemcpyHostToDevice, s));
+  BBO_CUDA(h, cudaMemcpyAsync(h->fits.p, fits.data(), sizeof(int2) * (size_t)n_fits, cudaMemcpyHostToDevice, s));
+  float* trace = nullptr;
+  if (tracing) {
+    const size_t cnt = (size_t)n_fits * h->opt.trace_steps;
+    BBO_CUDA(h, h->trace.reserve(cnt));
+    BBO_CUDA(h, cudaMemsetAsync(h->trace.p, 0xFF, cnt * sizeof(float), s));  // NaN padding
+    trace = h->trace.p;
+  }
+  float* keep = nullptr;
+  int64_t theta_count = 0;
+  if (h->opt.keep_theta) {
+    const int H = configs[n_configs - 1].hidden;
+    theta_count = (int64_t)d * H + H + (int64_t)H * C + C;
+    BBO_CUDA(h, h->theta.reserve((size_t)theta_count));
+    keep = h->theta.p;
+  }
+
+  BBO_CUDA(h, cudaEventRecord(h->ev0, s));
+  const float* Xk = X;
+  if (plan.dp != d || (reinterpret_cast<uintptr_t>(X) & 15u) != 0) {
+    BBO_CUDA(h, h->xpad.reserve((size_t)n * plan.dp));
+    const size_t total = (size_t)n * plan.dp;
+    bbo::pad_rows_kernel<<<(int)std::min<size_t>(1024, (total + 255) / 256), 256, 0, s>>>(X, n, d, plan.dp, h->xpad.p);
+    BBO_CUDA(h, cudaGetLastError());
+    ++launches;
+    Xk = h->xpad.p;
+  }
+  BBO_CUDA(h, launch_fold_permutation(n, seed, h->pi.p, s));
+  ++launches;
+
+  bbo::FitArgs a{};
+  a.X = Xk; a.y = y; a.pi = h->pi.p; a.configs = h->configs.p; a.fits = h->fits.p;
+  a.fold_scores = h->fold_scores.p; a.trace = trace; a.keep_theta = keep; a.queue = h->misc.p;
+  a.n_fits = n_fits; a.n_configs = n_configs;
+  a.n = n; a.d = d; a.dp = plan.dp; a.C = C; a.CS = plan.CS; a.K = K; a.task = task;
+  a.TB = plan.TB; a.trace_steps = h->opt.trace_steps; a.loss_cap = plan.loss_cap;
+  a.order_bytes = plan.order_bytes; a.seed = seed;
+  BBO_CUDA(h, launch_fit_any(C, a, h->sm_count, plan.NT, plan.smem, s));
+  ++launches;
+  bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(h->fold_scores.p, n_configs, K, out_scores);
+  BBO_CUDA(h, cudaGetLastError());
+  ++launches;
+  BBO_CUDA(h, cudaEventRecord(h->ev1, s));
+  BBO_CUDA(h, cudaStreamSynchronize(s));
+  BBO_CUDA(h, cudaEventElapsedTime(&h->last_ms, h->ev0, h->ev1));
+  h->last_launches = launches;
+  h->last_fold_count = n_fits;
+  h->last_trace_count = tracing ? (int64_t)n_fits * h->opt.trace_steps : 0;
+  h->last_theta_count = theta_count;
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_eval_host(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
+                         int32_t K, const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed,
+                         float* out_scores) {
+  if (!h || !X || !y || !configs || !out_scores || n < 2 || d < 1 || n_configs < 1) return BBO_ERR_INVALID_ARG;
+  if (n > kMaxRows) return BBO_ERR_UNSUPPORTED;
+  DeviceGuard g(h->device);
+  BBO_CUDA(h, h->hx.reserve((size_t)n * d));
+  BBO_CUDA(h, h->hy.reserve((size_t)n));
+  BBO_CUDA(h, h->hscores.reserve((size_t)n_configs));
+  BBO_CUDA(h, cudaMemcpyAsync(h->hx.p, X, sizeof(float) * (size_t)n * d, cudaMemcpyHostToDevice, h->stream));
+  BBO_CUDA(h, cudaMemcpyAsync(h->hy.p, y, sizeof(float) * (size_t)n, cudaMemcpyHostToDevice, h->stream));
+  const int rc = bbo_mlp_cv_eval(h, h->hx.p, h->hy.p, n, d, task, K, configs, n_configs, seed, h->hscores.p);
+  if (rc != BBO_OK) return rc;
+  BBO_CUDA(h, cudaMemcpyAsync(out_scores, h->hscores.p, sizeof(float) * (size_t)n_configs, cudaMemcpyDeviceToHost, h->stream));
+  BBO_CUDA(h, cudaStreamSynchronize(h->stream));
+  return BBO_OK;
+}
+
+static int copy_back(bbo_mlp_cv* h, const float* src, int64_t have, float* host_out, int64_t count) {
+  if (!h || !host_out) return BBO_ERR_INVALID_ARG;
+  if (have == 0 || count != have) return BBO_ERR_INVALID_ARG;
+  DeviceGuard g(h->device);
+  BBO_CUDA(h, cudaMemcpyAsync(host_out, src, sizeof(float) * (size_t)count, cudaMemcpyDeviceToHost, h->stream));
+  BBO_CUDA(h, cudaStreamSynchronize(h->stream));
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_fold_scores(bbo_mlp_cv* h, float* host_out, int64_t count) {
+  return h ? copy_back(h, h->fold_scores.p, h->last_fold_count, host_out, count) : BBO_ERR_INVALID_ARG;
+}
+int bbo_mlp_cv_loss_trace(bbo_mlp_cv* h, float* host_out, int64_t count) {
+  return h ? copy_back(h, h->trace.p, h->last_trace_count, host_out, count) : BBO_ERR_INVALID_ARG;
+}
+int bbo_mlp_cv_debug_theta(bbo_mlp_cv* h, float* host_out, int64_t count) {
+  return h ? copy_back(h, h->theta.p, h->last_theta_count, host_out, count) : BBO_ERR_INVALID_ARG;
+}
+
+int bbo_mlp_cv_debug_indices(bbo_mlp_cv* h, int64_t n64, int32_t K, uint64_t seed, int32_t config, int32_t fold,
+                             int32_t epoch, int32_t* host_fold_of_row, int32_t* host_order) {
+  if (!h || n64 < 2 || K < 2 || K > n64 || fold < 0 || fold >= K || config < 0 || epoch < 0) return BBO_ERR_INVALID_ARG;
+  if (n64 > kMaxRows || n64 > 65535) return BBO_ERR_UNSUPPORTED;
+  const int n = (int)n64;
+  DeviceGuard g(h->device);
+  cudaStream_t s = h->stream;
+  BBO_CUDA(h, h->pi.reserve(n));
+  BBO_CUDA(h, h->dbg_i.reserve(2 * (size_t)n));
+  BBO_CUDA(h, launch_fold_permutation(n, seed, h->pi.p, s));
+  int vb, vs;
+  bbo::fold_segment(n, K, fold, &vb, &vs);
+  const int n_tr = n - vs;
+  const size_t bytes = (size_t)bbo::round_up(2 * n_tr, 16) + 8u * (size_t)bbo::next_pow2(n_tr);
+  BBO_CUDA(h, cudaFuncSetAttribute(bbo::debug_order_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+  bbo::debug_order_kernel<<<1, 256, bytes, s>>>(n, K, seed, h->pi.p, config, fold, epoch, h->dbg_i.p, h->dbg_i.p + n);
+  BBO_CUDA(h, cudaGetLastError());
+  if (host_fold_of_row)
+    BBO_CUDA(h, cudaMemcpyAsync(host_fold_of_row, h->dbg_i.p, sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToHost, s));
+  if (host_order)
+    BBO_CUDA(h, cudaMemcpyAsync(host_order, h->dbg_i.p + n, sizeof(int32_t) * (size_t)n_tr, cudaMemcpyDeviceToHost, s));
+  BBO_CUDA(h, cudaStreamSynchronize(s));
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_debug_rng(bbo_mlp_cv* h, uint64_t seed, const uint32_t* counters, int64_t count, uint32_t* out) {
+  if (!h || !counters || !out || count < 1) return BBO_ERR_INVALID_ARG;
+  DeviceGuard g(h->device);
+  cudaStream_t s = h->stream;
+  BBO_CUDA(h, h->dbg_u.reserve(9 * (size_t)count));
+  BBO_CUDA(h, cudaMemcpyAsync(h->dbg_u.p, counters, sizeof(uint32_t) * 5 * (size_t)count, cudaMemcpyHostToDevice, s));
+  bbo::debug_rng_kernel<<<(int)std::min<int64_t>(1024, (count + 255) / 256), 256, 0, s>>>(seed, h->dbg_u.p, count, h->dbg_u.p + 5 * count);
+  BBO_CUDA(h, cudaGetLastError());
+  BBO_CUDA(h, cudaMemcpyAsync(out, h->dbg_u.p + 5 * count, sizeof(uint32_t) * 4 * (size_t)count, cudaMemcpyDeviceToHost, s));
+  BBO_CUDA(h, cudaStreamSynchronize(s));
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* out) {
+  if (!h || !x || !out || count < 1) return BBO_ERR_INVALID_ARG;
+  DeviceGuard g(h->device);
+  cudaStream_t s = h->stream;
+  BBO_CUDA(h, h->dbg_f.reserve(2 * (size_t)count));
+  BBO_CUDA(h, cudaMemcpyAsync(h->dbg_f.p, x, sizeof(float) * (size_t)count, cudaMemcpyHostToDevice, s));
+  bbo::debug_exp_kernel<<<(int)std::min<int64_t>(1024, (count + 255) / 256), 256, 0, s>>>(h->dbg_f.p, count, h->dbg_f.p + count);
+  BBO_CUDA(h, cudaGetLastError());
+  BBO_CUDA(h, cudaMemcpyAsync(out, h->dbg_f.p + count, sizeof(float) * (size_t)count, cudaMemcpyDeviceToHost, s));
+  BBO_CUDA(h, cudaStreamSynchronize(s));
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* max_n, int32_t* max_d,
+                          int32_t* max_hidden, int32_t* max_classes) {
+  if (!h || d < 1 || n_classes < 1 || n_classes > kMaxClasses) return BBO_ERR_INVALID_ARG;
+  if (max_n) *max_n = kMaxRows;
+  if (max_classes) *max_classes = kMaxClasses;
+  // widest hidden layer for (d, C) on a 1797-row, 5-fold problem with the smallest sub-tile
+  auto fits_H = [&](int dd, int H) {
+    Plan p;
+    return plan_launch(h, 1797, dd, n_classes, 5, H, 1, false, &p) == BBO_OK;
+  };
+  if (max_hidden) {
+    int lo = 0, hi = 4096;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) / 2;
+      if (fits_H(d, mid)) lo = mid; else hi = mid - 1;
+    }
+    *max_hidden = lo;
+  }
+  if (max_d) {
+    int lo = 0, hi = 16384;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) / 2;
+      if (fits_H(mid, 1)) lo = mid; else hi = mid - 1;
+    }
+    *max_d = lo;
+  }
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* kernel_ms, int32_t* n_launches) {
+  if (!h) return BBO_ERR_INVALID_ARG;
+  if (kernel_ms) *kernel_ms = h->last_ms;
+  if (n_launches) *n_launches = h->last_launches;
+  return BBO_OK;
+}
+
+const char* bbo_mlp_cv_strerror(int code) {
+  switch (code) {
+    case BBO_OK: return "ok";
+    case BBO_ERR_INVALID_ARG: return "invalid argument";
+    case BBO_ERR_UNSUPPORTED: return "shape or device not supported";
+    case BBO_ERR_CUDA: return "CUDA runtime error";
+    case BBO_ERR_TIMEOUT: return "device-side wait timed out";
+    case BBO_ERR_OOM: return "out of device memory";
+    default: return "unknown status";
+  }
+}
+
+const char* bbo_mlp_cv_last_cuda_error(bbo_mlp_cv* h) { return h ? h->cuda_error.c_str() : ""; }
+
+}  // extern "C"
