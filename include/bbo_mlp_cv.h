@@ -126,9 +126,11 @@ int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* ou
 int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* max_n,
                           int32_t* max_d, int32_t* max_hidden, int32_t* max_classes);
 
-/* Device time of the last eval's kernels (fold split .. fold mean) in milliseconds, and the
- * number of kernels it launched.  Either pointer may be NULL.                             */
-int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* kernel_ms, int32_t* n_launches);
+/* Device time (CUDA events on the handle's stream) of the last eval in milliseconds:
+ * total_ms from before the first kernel (row padding / fold permutation) to after the fold
+ * mean, fit_ms around the fit kernel alone; and the number of kernels the eval launched.
+ * Any pointer may be NULL.                                                                */
+int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* total_ms, float* fit_ms, int32_t* n_launches);
 
 const char* bbo_mlp_cv_strerror(int code);
 /* Text of the last CUDA error seen by this handle ("" if none).  Valid until the next call. */

@@ -74,7 +74,7 @@ def load():
     L.bbo_mlp_cv_debug_rng.argtypes = [vp, u64, vp, i64, vp]
     L.bbo_mlp_cv_debug_exp.argtypes = [vp, vp, i64, vp]
     L.bbo_mlp_cv_query_caps.argtypes = [vp, i32, i32, vp, vp, vp, vp]
-    L.bbo_mlp_cv_last_timing.argtypes = [vp, vp, vp]
+    L.bbo_mlp_cv_last_timing.argtypes = [vp, vp, vp, vp]
     L.bbo_mlp_cv_strerror.argtypes = [ctypes.c_int]
     L.bbo_mlp_cv_strerror.restype = ctypes.c_char_p
     L.bbo_mlp_cv_last_cuda_error.argtypes = [vp]
@@ -217,9 +217,10 @@ class MlpCv:
         return dict(max_n=v[0].value, max_d=v[1].value, max_hidden=v[2].value, max_classes=v[3].value)
 
     def last_timing(self):
-        ms, nl = ctypes.c_float(), ctypes.c_int32()
-        self._check(load().bbo_mlp_cv_last_timing(self._h, ctypes.byref(ms), ctypes.byref(nl)))
-        return ms.value, nl.value
+        """(total_ms, fit_kernel_ms, kernels launched) of the last eval, from CUDA events."""
+        ms, fit, nl = ctypes.c_float(), ctypes.c_float(), ctypes.c_int32()
+        self._check(load().bbo_mlp_cv_last_timing(self._h, ctypes.byref(ms), ctypes.byref(fit), ctypes.byref(nl)))
+        return ms.value, fit.value, nl.value
 
     def close(self):
         if self._h is not None:

@@ -57,10 +57,10 @@ struct bbo_mlp_cv {
   DevBuf<float> fold_scores, trace, theta, xpad, hx, hy, hscores, dbg_f;
   DevBuf<int32_t> pi, misc, dbg_i;
   DevBuf<uint32_t> dbg_u;
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr, evf0 = nullptr, evf1 = nullptr;
   // last eval
   int64_t last_fold_count = 0, last_trace_count = 0, last_theta_count = 0;
-  float last_ms = 0.f;
+  float last_ms = 0.f, last_fit_ms = 0.f;
   int last_launches = 0;
 };
 
@@ -222,7 +222,8 @@ int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out) {
   h->sm_count = prop.multiProcessorCount;
   h->smem_optin = (int)prop.sharedMemPerBlockOptin;
   DeviceGuard g(dev);
-  if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess) {
+  if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess ||
+      cudaEventCreate(&h->evf0) != cudaSuccess || cudaEventCreate(&h->evf1) != cudaSuccess) {
     delete h;
     return BBO_ERR_CUDA;
   }
@@ -239,6 +240,8 @@ int bbo_mlp_cv_destroy(bbo_mlp_cv* h) {
   h->dbg_f.release(); h->pi.release(); h->misc.release(); h->dbg_i.release(); h->dbg_u.release();
   if (h->ev0) cudaEventDestroy(h->ev0);
   if (h->ev1) cudaEventDestroy(h->ev1);
+  if (h->evf0) cudaEventDestroy(h->evf0);
+  if (h->evf1) cudaEventDestroy(h->evf1);
   delete h;
   return BBO_OK;
 }
@@ -350,7 +353,9 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   a.n = n; a.d = d; a.dp = plan.dp; a.C = C; a.CS = plan.CS; a.K = K; a.task = task;
   a.TB = plan.TB; a.trace_steps = h->opt.trace_steps; a.loss_cap = plan.loss_cap;
   a.order_bytes = plan.order_bytes; a.seed = seed;
+  BBO_CUDA(h, cudaEventRecord(h->evf0, s));
   BBO_CUDA(h, launch_fit_any(C, a, h->sm_count, plan.NT, plan.smem, s));
+  BBO_CUDA(h, cudaEventRecord(h->evf1, s));
   ++launches;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(h->fold_scores.p, n_configs, K, out_scores);
   BBO_CUDA(h, cudaGetLastError());
@@ -358,6 +363,7 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   BBO_CUDA(h, cudaEventRecord(h->ev1, s));
   BBO_CUDA(h, cudaStreamSynchronize(s));
   BBO_CUDA(h, cudaEventElapsedTime(&h->last_ms, h->ev0, h->ev1));
+  BBO_CUDA(h, cudaEventElapsedTime(&h->last_fit_ms, h->evf0, h->evf1));
   h->last_launches = launches;
   h->last_fold_count = n_fits;
   h->last_trace_count = tracing ? (int64_t)n_fits * h->opt.trace_steps : 0;
@@ -482,9 +488,10 @@ int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* 
   return BBO_OK;
 }
 
-int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* kernel_ms, int32_t* n_launches) {
+int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* total_ms, float* fit_ms, int32_t* n_launches) {
   if (!h) return BBO_ERR_INVALID_ARG;
-  if (kernel_ms) *kernel_ms = h->last_ms;
+  if (total_ms) *total_ms = h->last_ms;
+  if (fit_ms) *fit_ms = h->last_fit_ms;
   if (n_launches) *n_launches = h->last_launches;
   return BBO_OK;
 }
