@@ -52,7 +52,8 @@ typedef enum {
   BBO_ERR_UNSUPPORTED = -2, /* shape above the kernel caps, or not an sm_100 device         */
   BBO_ERR_CUDA = -3,        /* a CUDA runtime call failed (see bbo_mlp_cv_last_cuda_error)  */
   BBO_ERR_TIMEOUT = -4,     /* a bounded device-side wait gave up                           */
-  BBO_ERR_OOM = -5          /* scratch allocation failed                                    */
+  BBO_ERR_OOM = -5,         /* scratch allocation failed                                    */
+  BBO_ERR_TOO_LARGE = -6    /* problem exceeds the fixed scratch of bbo_mlp_cv_eval_static  */
 } bbo_status;
 
 /* Create-time options; a zeroed struct selects the defaults. */
@@ -131,6 +132,45 @@ int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* 
  * mean, fit_ms around the fit kernel alone; and the number of kernels the eval launched.
  * Any pointer may be NULL.                                                                */
 int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* total_ms, float* fit_ms, int32_t* n_launches);
+
+/* Allocation-free evaluation.  (The paper has no counterpart to this call; it exists for
+ * the library's users.)  Same result as bbo_mlp_cv_eval, for callers that must not allocate
+ * device memory while they run: code inside a memory-pool or arena framework that owns the
+ * whole device heap, real-time or latency-bound loops where cudaMalloc's implicit device
+ * synchronisation and unbounded latency are not acceptable, and processes that have already
+ * handed all free memory to another component.  It needs no handle, and it calls neither
+ * cudaMalloc nor cudaFree nor any allocating library routine.
+ *
+ * All working memory (fold permutation, device copy of the configurations, fit list,
+ * per-fold scores, work counter, padded copy of X) lives in ONE fixed array of
+ * BBO_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
+ * library holds those bytes until the process exits, used or not.  Hence the limits, checked
+ * before anything is enqueued and reported as BBO_ERR_TOO_LARGE:
+ *     n <= BBO_STATIC_MAX_ROWS,  n * roundup4(d) <= BBO_STATIC_MAX_X_FLOATS,
+ *     n_configs <= BBO_STATIC_MAX_CONFIGS,  n_configs * n_folds <= BBO_STATIC_MAX_FITS.
+ * Shapes above the kernel caps are BBO_ERR_UNSUPPORTED as in bbo_mlp_cv_eval.
+ *
+ *   stream     cudaStream_t of the CURRENT device (NULL = default stream); work is enqueued
+ *              there and the stream is synchronised before returning
+ *   X, y, out_scores  DEVICE buffers of the current device, as in bbo_mlp_cv_eval
+ *   n_classes  classification: 0 = 1 + max(y) found on the device; ignored for regression
+ *   configs    HOST [n_configs]
+ *
+ * The first call on each device looks up the array's device address and the device's
+ * limits (a one-off set-up, cached per device); make that first call before starting any
+ * stream capture.  The array is shared by every call in the process and keeps the previous
+ * call's contents; the call clears what has to start from zero.  Two calls that overlap on
+ * the same GPU (different streams or threads) would race on it: run them one after another. */
+#define BBO_STATIC_MAX_ROWS 4096
+#define BBO_STATIC_MAX_X_FLOATS 262144
+#define BBO_STATIC_MAX_CONFIGS 4096
+#define BBO_STATIC_MAX_FITS 16384
+#define BBO_STATIC_SCRATCH_BYTES (256 + 4 * BBO_STATIC_MAX_ROWS + 32 * BBO_STATIC_MAX_CONFIGS + \
+                                  12 * BBO_STATIC_MAX_FITS + 4 * BBO_STATIC_MAX_X_FLOATS)
+int bbo_mlp_cv_eval_static(void* stream, const float* X, const float* y, int64_t n, int32_t d,
+                           int32_t task, int32_t n_folds, int32_t n_classes,
+                           const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed,
+                           float* out_scores);
 
 const char* bbo_mlp_cv_strerror(int code);
 /* Text of the last CUDA error seen by this handle ("" if none).  Valid until the next call. */

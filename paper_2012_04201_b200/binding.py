@@ -22,6 +22,7 @@ BBO_ERR_UNSUPPORTED = -2
 BBO_ERR_CUDA = -3
 BBO_ERR_TIMEOUT = -4
 BBO_ERR_OOM = -5
+BBO_ERR_TOO_LARGE = -6
 
 TASK_CLASSIFICATION = 0
 TASK_REGRESSION = 1
@@ -31,7 +32,7 @@ EXPORTS = [
     "bbo_mlp_cv_fold_scores", "bbo_mlp_cv_loss_trace", "bbo_mlp_cv_debug_theta",
     "bbo_mlp_cv_debug_indices", "bbo_mlp_cv_debug_rng", "bbo_mlp_cv_debug_exp",
     "bbo_mlp_cv_query_caps", "bbo_mlp_cv_last_timing", "bbo_mlp_cv_strerror",
-    "bbo_mlp_cv_last_cuda_error",
+    "bbo_mlp_cv_last_cuda_error", "bbo_mlp_cv_eval_static",
 ]
 
 
@@ -67,6 +68,7 @@ def load():
     L.bbo_mlp_cv_eval.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_eval_host.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_destroy.argtypes = [vp]
+    L.bbo_mlp_cv_eval_static.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_fold_scores.argtypes = [vp, vp, i64]
     L.bbo_mlp_cv_loss_trace.argtypes = [vp, vp, i64]
     L.bbo_mlp_cv_debug_theta.argtypes = [vp, vp, i64]
@@ -123,6 +125,16 @@ def bbo_mlp_cv_eval_host(h, X, y, task, n_folds, configs, seed, out):
 
 def bbo_mlp_cv_destroy(h):
     return load().bbo_mlp_cv_destroy(h)
+
+
+def bbo_mlp_cv_eval_static(stream_ptr, X_ptr, y_ptr, n, d, task, n_folds, n_classes, configs, seed, out_ptr):
+    """Allocation-free evaluation on the current device (no handle).  Device pointers (ints)
+    for X, y, out; ``configs`` a CONFIG_DTYPE array.  All device scratch comes from a fixed
+    array inside the library, so the call never asks the driver for memory; problems above
+    the documented limits return BBO_ERR_TOO_LARGE.  Returns the status code."""
+    configs = np.ascontiguousarray(configs, dtype=CONFIG_DTYPE)
+    return load().bbo_mlp_cv_eval_static(stream_ptr or None, X_ptr, y_ptr, n, d, task, n_folds, n_classes,
+                                         _np_ptr(configs), configs.size, seed, out_ptr)
 
 
 # ---- convenience wrapper ---------------------------------------------------------------

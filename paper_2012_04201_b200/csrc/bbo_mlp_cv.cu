@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -504,6 +505,7 @@ const char* bbo_mlp_cv_strerror(int code) {
     case BBO_ERR_CUDA: return "CUDA runtime error";
     case BBO_ERR_TIMEOUT: return "device-side wait timed out";
     case BBO_ERR_OOM: return "out of device memory";
+    case BBO_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the allocation-free entry point";
     default: return "unknown status";
   }
 }
@@ -511,3 +513,153 @@ const char* bbo_mlp_cv_strerror(int code) {
 const char* bbo_mlp_cv_last_cuda_error(bbo_mlp_cv* h) { return h ? h->cuda_error.c_str() : ""; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free evaluation: every working buffer is carved out of one array that is part
+// of the library image.  In host code the name `g_static_scratch` is only a handle for the
+// runtime, not a device address; the address comes from cudaGetSymbolAddress, once per
+// device, and that pointer is what the kernels receive.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[BBO_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+struct StaticDevice {
+  bool ready = false;
+  unsigned char* base = nullptr;
+  int sm_count = 0, smem_optin = 0, major = 0;
+};
+constexpr int kMaxDevices = 64;
+StaticDevice g_static_dev[kMaxDevices];
+std::mutex g_static_mutex;
+
+// One-off set-up for the current device: device address of the scratch array and the
+// device limits the launch plan needs.
+int static_device_setup(int dev, StaticDevice* out) {
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticDevice& sd = g_static_dev[dev];
+  if (!sd.ready) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+      cudaGetLastError();
+      return BBO_ERR_CUDA;
+    }
+    if (cudaDeviceGetAttribute(&sd.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sd.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sd.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return BBO_ERR_CUDA;
+    }
+    sd.base = static_cast<unsigned char*>(ptr);
+    sd.ready = true;
+  }
+  *out = sd;
+  return BBO_OK;
+}
+
+}  // namespace
+
+extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float* y, int64_t n64, int32_t d,
+                                      int32_t task, int32_t K, int32_t n_classes, const bbo_mlp_config* configs,
+                                      int32_t n_configs, uint64_t seed, float* out_scores) {
+  if (!X || !y || !configs || !out_scores) return BBO_ERR_INVALID_ARG;
+  if (n64 < 2 || d < 1 || K < 2 || K > n64 || n_configs < 1 || n_classes < 0 || n_classes > kMaxClasses)
+    return BBO_ERR_INVALID_ARG;
+  if (task != BBO_TASK_CLASSIFICATION && task != BBO_TASK_REGRESSION) return BBO_ERR_INVALID_ARG;
+  const int64_t dp64 = (int64_t)(d + 3) / 4 * 4;
+  if (n64 > BBO_STATIC_MAX_ROWS || n64 * dp64 > BBO_STATIC_MAX_X_FLOATS || n_configs > BBO_STATIC_MAX_CONFIGS ||
+      (int64_t)n_configs * K > BBO_STATIC_MAX_FITS)
+    return BBO_ERR_TOO_LARGE;
+  int maxH, maxB;
+  int rc = check_configs(configs, n_configs, &maxH, &maxB);
+  if (rc != BBO_OK) return rc;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BBO_ERR_CUDA;
+  StaticDevice sd;
+  rc = static_device_setup(dev, &sd);
+  if (rc != BBO_OK) return rc;
+  if (sd.major != 10) return BBO_ERR_UNSUPPORTED;
+  if (!is_device_ptr(X, dev) || !is_device_ptr(y, dev) || !is_device_ptr(out_scores, dev)) return BBO_ERR_INVALID_ARG;
+  const int n = (int)n64;
+  const int n_fits = n_configs * K;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  // carve the array: [misc 256 B][pi][configs][fits][fold scores][padded X]
+  unsigned char* p = sd.base;
+  int32_t* misc = reinterpret_cast<int32_t*>(p);            p += 256;
+  int32_t* pi = reinterpret_cast<int32_t*>(p);              p += 4 * (size_t)BBO_STATIC_MAX_ROWS;
+  bbo::Config* dcfg = reinterpret_cast<bbo::Config*>(p);    p += 32 * (size_t)BBO_STATIC_MAX_CONFIGS;
+  int2* dfits = reinterpret_cast<int2*>(p);                 p += 8 * (size_t)BBO_STATIC_MAX_FITS;
+  float* fold_scores = reinterpret_cast<float*>(p);         p += 4 * (size_t)BBO_STATIC_MAX_FITS;
+  float* xpad = reinterpret_cast<float*>(p);
+
+  // the work counter and the label summary must start from zero; everything else is
+  // fully rewritten before it is read
+  if (cudaMemsetAsync(misc, 0, 256, s) != cudaSuccess) return BBO_ERR_CUDA;
+  int C = 1;
+  if (task == BBO_TASK_CLASSIFICATION) {
+    bbo::label_scan_kernel<<<std::min(64, (n + 255) / 256), 256, 0, s>>>(y, n, misc + 1);
+    int32_t info[2];
+    if (cudaGetLastError() != cudaSuccess ||
+        cudaMemcpyAsync(info, misc + 1, sizeof(info), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+      return BBO_ERR_CUDA;
+    if (info[1] != 0) return BBO_ERR_INVALID_ARG;
+    C = info[0] + 1;
+    if (n_classes > 0) {
+      if (C > n_classes) return BBO_ERR_INVALID_ARG;
+      C = n_classes;
+    }
+    if (C > kMaxClasses) return BBO_ERR_UNSUPPORTED;
+  }
+
+  bbo_mlp_cv limits;  // only carries the device's shared-memory limit into the planner
+  limits.smem_optin = sd.smem_optin;
+  Plan plan;
+  rc = plan_launch(&limits, n, d, C, K, maxH, maxB, false, &plan);
+  if (rc != BBO_OK) return rc;
+
+  // fit list, costliest first (same ordering rule as bbo_mlp_cv_eval; host memory only)
+  std::vector<int2> fits((size_t)n_fits);
+  {
+    std::vector<std::pair<double, int>> cost((size_t)n_fits);
+    for (int c = 0; c < n_configs; ++c) {
+      const bbo_mlp_config& q = configs[c];
+      for (int f = 0; f < K; ++f) {
+        int vb, vs;
+        bbo::fold_segment(n, K, f, &vb, &vs);
+        const double n_tr = n - vs, B = std::min<double>(q.batch_size, n_tr);
+        const double P = (double)d * q.hidden + q.hidden + (double)q.hidden * C + C;
+        const double steps = (double)q.epochs * std::ceil(n_tr / B);
+        cost[(size_t)c * K + f] = {(double)q.epochs * n_tr * (4.0 * d * q.hidden + 6.0 * q.hidden * C) + steps * 14.0 * P,
+                                   c * K + f};
+      }
+    }
+    std::stable_sort(cost.begin(), cost.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
+    for (int i = 0; i < n_fits; ++i) fits[i] = make_int2(cost[i].second / K, cost[i].second % K);
+  }
+  if (cudaMemcpyAsync(dcfg, configs, sizeof(bbo_mlp_config) * (size_t)n_configs, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dfits, fits.data(), sizeof(int2) * (size_t)n_fits, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return BBO_ERR_CUDA;
+
+  const float* Xk = X;
+  if (plan.dp != d || (reinterpret_cast<uintptr_t>(X) & 15u) != 0) {
+    const size_t total = (size_t)n * plan.dp;
+    bbo::pad_rows_kernel<<<(int)std::min<size_t>(1024, (total + 255) / 256), 256, 0, s>>>(X, n, d, plan.dp, xpad);
+    if (cudaGetLastError() != cudaSuccess) return BBO_ERR_CUDA;
+    Xk = xpad;
+  }
+  if (launch_fold_permutation(n, seed, pi, s) != cudaSuccess) return BBO_ERR_CUDA;
+
+  bbo::FitArgs a{};
+  a.X = Xk; a.y = y; a.pi = pi; a.configs = dcfg; a.fits = dfits;
+  a.fold_scores = fold_scores; a.trace = nullptr; a.keep_theta = nullptr; a.queue = misc;
+  a.n_fits = n_fits; a.n_configs = n_configs;
+  a.n = n; a.d = d; a.dp = plan.dp; a.C = C; a.CS = plan.CS; a.K = K; a.task = task;
+  a.TB = plan.TB; a.trace_steps = 0; a.loss_cap = plan.loss_cap;
+  a.order_bytes = plan.order_bytes; a.seed = seed;
+  if (launch_fit_any(C, a, sd.sm_count, plan.NT, plan.smem, s) != cudaSuccess) return BBO_ERR_CUDA;
+  bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(fold_scores, n_configs, K, out_scores);
+  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return BBO_ERR_CUDA;
+  return BBO_OK;
+}
