@@ -1,0 +1,73 @@
+// Small kernels around the fit kernel: fold permutation, fold mean, label scan, row padding
+// and the debug exports.  Included by exactly one translation unit.
+#pragma once
+#include "fit_common.cuh"
+
+namespace bbo {
+
+// Fold split: pi = permutation of the rows by ascending (random word << 32 | row).
+__global__ void fold_permutation_kernel(int n, uint64_t seed, int32_t* pi) {
+  extern __shared__ __align__(16) float smem[];
+  uint64_t* keys = reinterpret_cast<uint64_t*>(smem);
+  sorted_keys(keys, n, seed, kStreamFold, 0u, 0u, 0u, threadIdx.x, blockDim.x);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) pi[i] = (int32_t)(uint32_t)keys[i];
+}
+
+// out[c] = (score[c][0] + ... + score[c][K-1]) / K, ascending fold.
+__global__ void fold_mean_kernel(const float* fold_scores, int n_configs, int K, float* out) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= n_configs) return;
+  float s = 0.f;
+  for (int f = 0; f < K; ++f) s = __fadd_rn(s, fold_scores[(size_t)c * K + f]);
+  out[c] = __fdiv_rn(s, (float)K);
+}
+
+// info[0] = max label, info[1] = 1 if any label is negative, fractional, huge or NaN.
+__global__ void label_scan_kernel(const float* y, int n, int32_t* info) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const float v = y[i];
+    if (!(v >= 0.f) || v != floorf(v) || v > 1.0e6f) atomicOr(&info[1], 1);
+    else atomicMax(&info[0], (int)v);
+  }
+}
+
+// Copy X into rows of dp floats (zero padded) so that every row starts 16-byte aligned.
+__global__ void pad_rows_kernel(const float* X, int n, int d, int dp, float* out) {
+  const size_t total = (size_t)n * dp;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / dp), k = (int)(i - (size_t)r * dp);
+    out[i] = k < d ? X[(size_t)r * d + k] : 0.f;
+  }
+}
+
+// Debug: epoch order of one fit written to global memory, and the fold of every row.
+__global__ void debug_order_kernel(int n, int K, uint64_t seed, const int32_t* pi, int config, int fold,
+                                   int epoch, int32_t* fold_of_row, int32_t* order_out) {
+  extern __shared__ __align__(16) float smem[];
+  int vb, vs;
+  fold_segment(n, K, fold, &vb, &vs);
+  const int n_tr = n - vs;
+  uint16_t* order = reinterpret_cast<uint16_t*>(smem);
+  uint64_t* keys = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(smem) + round_up(2 * n_tr, 16));
+  build_epoch_order(keys, order, pi, n_tr, vb, vs, seed, config, fold, epoch, threadIdx.x, blockDim.x);
+  for (int i = threadIdx.x; i < n_tr; i += blockDim.x) order_out[i] = order[i];
+  for (int f = 0; f < K; ++f) {
+    int b, s;
+    fold_segment(n, K, f, &b, &s);
+    for (int i = threadIdx.x; i < s; i += blockDim.x) fold_of_row[pi[b + i]] = f;
+  }
+}
+
+__global__ void debug_rng_kernel(uint64_t seed, const uint32_t* ctr, int64_t count, uint32_t* out) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+    const uint4 r = philox4x32_10(seed, ctr[5 * i], ctr[5 * i + 1], ctr[5 * i + 2], ctr[5 * i + 3], ctr[5 * i + 4]);
+    out[4 * i] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
+  }
+}
+
+__global__ void debug_exp_kernel(const float* x, int64_t count, float* out) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    out[i] = spec_expf(x[i]);
+}
+
+}  // namespace bbo

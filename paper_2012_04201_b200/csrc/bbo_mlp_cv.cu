@@ -12,14 +12,16 @@
 #include <vector>
 
 #include "../../include/bbo_mlp_cv.h"
-#include "fit_kernel.cuh"
+#include "aux_kernels.cuh"
+#include "fit_launch.h"
 
 static_assert(sizeof(bbo_mlp_config) == 32, "bbo_mlp_config must be 32 bytes");
 static_assert(sizeof(bbo::Config) == sizeof(bbo_mlp_config), "device mirror of bbo_mlp_config");
 
 namespace {
 
-constexpr int kMaxClasses = 16;
+using bbo::kMaxClasses;
+constexpr int kAuxStreams = 4;  // buckets of different hidden width overlap on these
 constexpr int kMaxThreads = 512;
 constexpr int kMaxRows = 16384;  // fold permutation sorts in one CTA's shared memory
 
@@ -59,6 +61,8 @@ struct bbo_mlp_cv {
   DevBuf<int32_t> pi, misc, dbg_i;
   DevBuf<uint32_t> dbg_u;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr, evf0 = nullptr, evf1 = nullptr;
+  cudaStream_t aux[kAuxStreams] = {};
+  cudaEvent_t fork = nullptr, join[kAuxStreams] = {};
   // last eval
   int64_t last_fold_count = 0, last_trace_count = 0, last_theta_count = 0;
   float last_ms = 0.f, last_fit_ms = 0.f;
@@ -99,76 +103,148 @@ bool is_device_ptr(const void* p, int device) {
   return (at.type == cudaMemoryTypeDevice && at.device == device) || at.type == cudaMemoryTypeManaged;
 }
 
+// Launch geometry of the fits that share one padded hidden width.
 struct Plan {
-  int C, CS, dp, TB, NT, order_bytes, loss_cap, n_sort;
+  int C, CS, dp, Hs, TB, NT, order_bytes, loss_cap, n_sort, per_sm;
+  bool vreg;
   size_t smem;
 };
 
-// Threads needed by a fit of width H: one per gradient tile (4 rows x 8 columns of W1) and
-// one per hidden unit.
-int threads_for(int dp, int H) {
-  const int Hs = bbo::round_up(H, 8);
-  const int tiles = (dp / 4) * (Hs / 8);
-  return bbo::round_up(std::max(std::max(tiles, Hs), 64), 32);
+// CTAs of `threads` threads and `smem` bytes that fit on one SM (registers: the kernels are
+// compiled for at most 128 per thread; warps are placed four at a time).
+int ctas_per_sm(int smem_total, int threads, size_t smem) {
+  const int by_smem = (int)((size_t)smem_total / (smem + 1024));
+  const int by_threads = 2048 / threads;
+  const int by_regs = 512 / bbo::round_up(threads, 128) ;
+  return std::max(0, std::min(by_smem, std::min(by_threads, by_regs)));
 }
 
-size_t smem_for(int d, int dp, int H, int CS, int TB, int order_bytes, int loss_cap, int n_sort) {
-  bbo::Layout L(d, H, CS);
-  return 3u * (size_t)L.PS * 4u + bbo::scratch_bytes(L.Hs, dp, CS, TB, order_bytes, loss_cap, n_sort);
-}
-
-// Largest sub-tile height (64, 32, ... 4) for which the widest fit fits in shared memory.
-int plan_launch(const bbo_mlp_cv* h, int n, int d, int C, int K, int maxH, int maxB, bool tracing, Plan* out) {
+// Plans the launch of fits of padded width Hs.  Threads: one per gradient tile of W1 (4 rows x
+// 8 columns) and two per hidden unit.  Sub-tile height: the largest of 32, 16, 8, 4 that fits.
+// The second moments of W1 move to registers when that lets more CTAs share an SM.
+int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bool tracing, Plan* out) {
   Plan p{};
   p.C = C;
   p.CS = bbo::round_up(C, 4);
   p.dp = bbo::round_up(d, 4);
+  p.Hs = Hs;
   const int n_tr_max = n - n / K;
   p.order_bytes = bbo::round_up(2 * n_tr_max, 16);
   p.loss_cap = tracing ? std::min(maxB, n_tr_max) : 0;
   p.n_sort = n_tr_max;
-  p.NT = threads_for(p.dp, maxH);
+  const int tiles = (p.dp / 4) * (Hs / 8);
+  p.NT = bbo::round_up(std::max(std::max(tiles, 2 * Hs), 64), 32);
   if (p.NT > kMaxThreads) return BBO_ERR_UNSUPPORTED;
-  const size_t budget = (size_t)h->smem_optin - 256;  // static block scalars
+  const size_t budget = (size_t)smem_optin - 256;  // static block scalars
+  const int smem_sm = smem_optin + 1024;
   for (int TB = 32; TB >= 4; TB >>= 1) {
-    const size_t need = smem_for(d, p.dp, maxH, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort);
-    if (need <= budget) {
-      p.TB = TB;
-      p.smem = need;
-      *out = p;
-      return BBO_OK;
-    }
+    const size_t plain = bbo::fit_smem_bytes(d, p.dp, Hs, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, false);
+    const size_t lean = bbo::fit_smem_bytes(d, p.dp, Hs, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
+    if (lean > budget) continue;
+    const int occ_plain = plain <= budget ? ctas_per_sm(smem_sm, p.NT, plain) : 0;
+    const int occ_lean = ctas_per_sm(smem_sm, p.NT, lean);
+    p.TB = TB;
+    p.vreg = occ_lean > occ_plain && p.NT <= 256;
+    if (!p.vreg && plain > budget) continue;
+    p.smem = p.vreg ? lean : plain;
+    p.per_sm = std::max(1, p.vreg ? occ_lean : occ_plain);
+    *out = p;
+    return BBO_OK;
   }
   return BBO_ERR_UNSUPPORTED;
 }
 
-template <typename Kern>
-cudaError_t launch_kernel(Kern kern, const bbo::FitArgs& a, int n_sm, int NT, size_t smem, cudaStream_t s) {
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NT, smem);
-  if (e != cudaSuccess) return e;
-  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  const int grid = std::min(a.n_fits, n_sm * per_sm);  // persistent CTAs, all resident
-  kern<<<grid, NT, smem, s>>>(a);
-  return cudaGetLastError();
-}
+// Where the fits of one evaluation run: the caller's stream plus optional side streams.
+struct LaunchEnv {
+  int smem_optin = 0;
+  cudaStream_t main = nullptr;
+  cudaStream_t* aux = nullptr;  // may be null: everything runs on `main`
+  int n_aux = 0;
+  cudaEvent_t fork = nullptr;
+  cudaEvent_t* join = nullptr;
+};
 
-template <int CT>
-cudaError_t launch_fit(const bbo::FitArgs& a, int n_sm, int NT, size_t smem, cudaStream_t s) {
-  if (NT <= 256) return launch_kernel(bbo::mlp_cv_fit_kernel<CT, 256>, a, n_sm, NT, smem, s);
-  return launch_kernel(bbo::mlp_cv_fit_kernel<CT, 512>, a, n_sm, NT, smem, s);
-}
+struct FitBuffers {  // device scratch of one evaluation
+  bbo::Config* configs;
+  int2* fits;
+  float* fold_scores;
+  const int32_t* pi;
+  float* trace;
+  float* keep_theta;
+};
 
-cudaError_t launch_fit_any(int C, const bbo::FitArgs& a, int n_sm, int NT, size_t smem, cudaStream_t s) {
-  switch (C) {
-    case 1: return launch_fit<1>(a, n_sm, NT, smem, s);
-    case 2: return launch_fit<2>(a, n_sm, NT, smem, s);
-    case 3: return launch_fit<3>(a, n_sm, NT, smem, s);
-    case 10: return launch_fit<10>(a, n_sm, NT, smem, s);
-    default: return C <= 4 ? launch_fit<4>(a, n_sm, NT, smem, s) : launch_fit<kMaxClasses>(a, n_sm, NT, smem, s);
+// Groups the fits by padded hidden width, orders each group by descending cost estimate
+// E * n_train * (4dH + 6HC) + steps * 14 P, uploads the lists and launches one grid per group
+// (widest first; groups overlap on the side streams when there are any).
+int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk, const float* y, int n, int d,
+                    int C, int K, int task, const bbo_mlp_config* configs, int n_configs, uint64_t seed,
+                    int trace_steps, int maxB, int* launches, cudaError_t* cuda_err) {
+  *cuda_err = cudaSuccess;
+  const int n_fits = n_configs * K;
+  struct Item { int Hs; double cost; int id; };
+  std::vector<Item> items((size_t)n_fits);
+  for (int c = 0; c < n_configs; ++c) {
+    const bbo_mlp_config& q = configs[c];
+    for (int f = 0; f < K; ++f) {
+      int vb, vs;
+      bbo::fold_segment(n, K, f, &vb, &vs);
+      const double n_tr = n - vs, B = std::min<double>(q.batch_size, n_tr);
+      const double P = (double)d * q.hidden + q.hidden + (double)q.hidden * C + C;
+      const double steps = (double)q.epochs * std::ceil(n_tr / B);
+      items[(size_t)c * K + f] = {bbo::round_up(q.hidden, 8),
+                                  (double)q.epochs * n_tr * (4.0 * d * q.hidden + 6.0 * q.hidden * C) + steps * 14.0 * P,
+                                  c * K + f};
+    }
   }
+  std::stable_sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
+    return a.Hs != b.Hs ? a.Hs > b.Hs : a.cost > b.cost;
+  });
+  std::vector<int2> fits((size_t)n_fits);
+  for (int i = 0; i < n_fits; ++i) fits[i] = make_int2(items[i].id / K, items[i].id % K);
+  // plan every group before anything is enqueued
+  struct Group { int begin, count; Plan plan; };
+  std::vector<Group> groups;
+  for (int i = 0; i < n_fits;) {
+    int j = i;
+    while (j < n_fits && items[j].Hs == items[i].Hs) ++j;
+    Group g{i, j - i, {}};
+    const int rc = plan_bucket(env.smem_optin, n, d, C, K, items[i].Hs, maxB, trace_steps > 0, &g.plan);
+    if (rc != BBO_OK) return rc;
+    groups.push_back(g);
+    i = j;
+  }
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(buf.configs, configs, sizeof(bbo_mlp_config) * (size_t)n_configs, cudaMemcpyHostToDevice, env.main)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(buf.fits, fits.data(), sizeof(int2) * (size_t)n_fits, cudaMemcpyHostToDevice, env.main)) != cudaSuccess) {
+    *cuda_err = e;
+    return BBO_ERR_CUDA;
+  }
+  const bool side = env.n_aux > 0 && groups.size() > 1;
+  if (side) {
+    if ((e = cudaEventRecord(env.fork, env.main)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
+    for (int i = 0; i < env.n_aux; ++i)
+      if ((e = cudaStreamWaitEvent(env.aux[i], env.fork, 0)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
+  }
+  for (size_t gi = 0; gi < groups.size(); ++gi) {
+    const Group& g = groups[gi];
+    bbo::FitArgs a{};
+    a.X = Xk; a.y = y; a.pi = buf.pi; a.configs = buf.configs; a.fits = buf.fits + g.begin;
+    a.fold_scores = buf.fold_scores; a.trace = buf.trace; a.keep_theta = buf.keep_theta;
+    a.n_fits = g.count; a.n_configs = n_configs;
+    a.n = n; a.d = d; a.dp = g.plan.dp; a.C = C; a.CS = g.plan.CS; a.K = K; a.task = task;
+    a.Hs = g.plan.Hs; a.TB = g.plan.TB; a.trace_steps = trace_steps; a.loss_cap = g.plan.loss_cap;
+    a.order_bytes = g.plan.order_bytes; a.seed = seed;
+    cudaStream_t s = side ? env.aux[gi % env.n_aux] : env.main;
+    if ((e = bbo::launch_fit(C, a, g.plan.vreg, g.plan.NT, g.count, g.plan.smem, s)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
+    ++*launches;
+  }
+  if (side) {
+    for (int i = 0; i < env.n_aux; ++i) {
+      if ((e = cudaEventRecord(env.join[i], env.aux[i])) != cudaSuccess ||
+          (e = cudaStreamWaitEvent(env.main, env.join[i], 0)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
+    }
+  }
+  return BBO_OK;
 }
 
 cudaError_t launch_fold_permutation(int n, uint64_t seed, int32_t* pi, cudaStream_t s) {
@@ -228,6 +304,14 @@ int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out) {
     delete h;
     return BBO_ERR_CUDA;
   }
+  bool ok = cudaEventCreateWithFlags(&h->fork, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < kAuxStreams && ok; ++i)
+    ok = cudaStreamCreateWithFlags(&h->aux[i], cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&h->join[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    bbo_mlp_cv_destroy(h);
+    return BBO_ERR_CUDA;
+  }
   *out = h;
   return BBO_OK;
 }
@@ -243,6 +327,11 @@ int bbo_mlp_cv_destroy(bbo_mlp_cv* h) {
   if (h->ev1) cudaEventDestroy(h->ev1);
   if (h->evf0) cudaEventDestroy(h->evf0);
   if (h->evf1) cudaEventDestroy(h->evf1);
+  if (h->fork) cudaEventDestroy(h->fork);
+  for (int i = 0; i < kAuxStreams; ++i) {
+    if (h->join[i]) cudaEventDestroy(h->join[i]);
+    if (h->aux[i]) cudaStreamDestroy(h->aux[i]);
+  }
   delete h;
   return BBO_OK;
 }
@@ -286,38 +375,13 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
     if (C > kMaxClasses) return BBO_ERR_UNSUPPORTED;
   }
 
-  Plan plan;
   const bool tracing = h->opt.trace_steps > 0;
-  rc = plan_launch(h, n, d, C, K, maxH, maxB, tracing, &plan);
-  if (rc != BBO_OK) return rc;
-
+  const int dp = bbo::round_up(d, 4);
   const int n_fits = n_configs * K;
-  // fit list, costliest first: E * n_train * (4dH + 6HC) + steps * 14 P
-  std::vector<int2> fits((size_t)n_fits);
-  {
-    std::vector<std::pair<double, int>> cost((size_t)n_fits);
-    for (int c = 0; c < n_configs; ++c) {
-      const bbo_mlp_config& q = configs[c];
-      for (int f = 0; f < K; ++f) {
-        int vb, vs;
-        bbo::fold_segment(n, K, f, &vb, &vs);
-        const double n_tr = n - vs, B = std::min<double>(q.batch_size, n_tr);
-        const double P = (double)d * q.hidden + q.hidden + (double)q.hidden * C + C;
-        const double steps = (double)q.epochs * std::ceil(n_tr / B);
-        cost[(size_t)c * K + f] = {(double)q.epochs * n_tr * (4.0 * d * q.hidden + 6.0 * q.hidden * C) + steps * 14.0 * P,
-                                   c * K + f};
-      }
-    }
-    std::stable_sort(cost.begin(), cost.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
-    for (int i = 0; i < n_fits; ++i) fits[i] = make_int2(cost[i].second / K, cost[i].second % K);
-  }
-
   BBO_CUDA(h, h->configs.reserve(n_configs));
   BBO_CUDA(h, h->fits.reserve(n_fits));
   BBO_CUDA(h, h->fold_scores.reserve(n_fits));
   BBO_CUDA(h, h->pi.reserve(n));
-  BBO_CUDA(h, cudaMemcpyAsync(h->configs.p, configs, sizeof(bbo_mlp_config) * (size_t)n_configs, cudaMemcpyHostToDevice, s));
-  BBO_CUDA(h, cudaMemcpyAsync(h->fits.p, fits.data(), sizeof(int2) * (size_t)n_fits, cudaMemcpyHostToDevice, s));
   float* trace = nullptr;
   if (tracing) {
     const size_t cnt = (size_t)n_fits * h->opt.trace_steps;
@@ -336,10 +400,10 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
 
   BBO_CUDA(h, cudaEventRecord(h->ev0, s));
   const float* Xk = X;
-  if (plan.dp != d || (reinterpret_cast<uintptr_t>(X) & 15u) != 0) {
-    BBO_CUDA(h, h->xpad.reserve((size_t)n * plan.dp));
-    const size_t total = (size_t)n * plan.dp;
-    bbo::pad_rows_kernel<<<(int)std::min<size_t>(1024, (total + 255) / 256), 256, 0, s>>>(X, n, d, plan.dp, h->xpad.p);
+  if (dp != d || (reinterpret_cast<uintptr_t>(X) & 15u) != 0) {
+    BBO_CUDA(h, h->xpad.reserve((size_t)n * dp));
+    const size_t total = (size_t)n * dp;
+    bbo::pad_rows_kernel<<<(int)std::min<size_t>(1024, (total + 255) / 256), 256, 0, s>>>(X, n, d, dp, h->xpad.p);
     BBO_CUDA(h, cudaGetLastError());
     ++launches;
     Xk = h->xpad.p;
@@ -347,17 +411,17 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   BBO_CUDA(h, launch_fold_permutation(n, seed, h->pi.p, s));
   ++launches;
 
-  bbo::FitArgs a{};
-  a.X = Xk; a.y = y; a.pi = h->pi.p; a.configs = h->configs.p; a.fits = h->fits.p;
-  a.fold_scores = h->fold_scores.p; a.trace = trace; a.keep_theta = keep; a.queue = h->misc.p;
-  a.n_fits = n_fits; a.n_configs = n_configs;
-  a.n = n; a.d = d; a.dp = plan.dp; a.C = C; a.CS = plan.CS; a.K = K; a.task = task;
-  a.TB = plan.TB; a.trace_steps = h->opt.trace_steps; a.loss_cap = plan.loss_cap;
-  a.order_bytes = plan.order_bytes; a.seed = seed;
+  LaunchEnv env;
+  env.smem_optin = h->smem_optin; env.main = s; env.aux = h->aux; env.n_aux = kAuxStreams;
+  env.fork = h->fork; env.join = h->join;
+  FitBuffers buf{h->configs.p, h->fits.p, h->fold_scores.p, h->pi.p, trace, keep};
   BBO_CUDA(h, cudaEventRecord(h->evf0, s));
-  BBO_CUDA(h, launch_fit_any(C, a, h->sm_count, plan.NT, plan.smem, s));
+  cudaError_t cuda_err = cudaSuccess;
+  rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, h->opt.trace_steps, maxB,
+                       &launches, &cuda_err);
+  if (rc == BBO_ERR_CUDA) return cuda_fail(h, cuda_err, "launch_all_fits");
+  if (rc != BBO_OK) return rc;
   BBO_CUDA(h, cudaEventRecord(h->evf1, s));
-  ++launches;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(h->fold_scores.p, n_configs, K, out_scores);
   BBO_CUDA(h, cudaGetLastError());
   ++launches;
@@ -468,7 +532,7 @@ int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* 
   // widest hidden layer for (d, C) on a 1797-row, 5-fold problem with the smallest sub-tile
   auto fits_H = [&](int dd, int H) {
     Plan p;
-    return plan_launch(h, 1797, dd, n_classes, 5, H, 1, false, &p) == BBO_OK;
+    return plan_bucket(h->smem_optin, 1797, dd, n_classes, 5, bbo::round_up(H, 8), 1, false, &p) == BBO_OK;
   };
   if (max_hidden) {
     int lo = 0, hi = 4096;
@@ -613,52 +677,23 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
     if (C > kMaxClasses) return BBO_ERR_UNSUPPORTED;
   }
 
-  bbo_mlp_cv limits;  // only carries the device's shared-memory limit into the planner
-  limits.smem_optin = sd.smem_optin;
-  Plan plan;
-  rc = plan_launch(&limits, n, d, C, K, maxH, maxB, false, &plan);
-  if (rc != BBO_OK) return rc;
-
-  // fit list, costliest first (same ordering rule as bbo_mlp_cv_eval; host memory only)
-  std::vector<int2> fits((size_t)n_fits);
-  {
-    std::vector<std::pair<double, int>> cost((size_t)n_fits);
-    for (int c = 0; c < n_configs; ++c) {
-      const bbo_mlp_config& q = configs[c];
-      for (int f = 0; f < K; ++f) {
-        int vb, vs;
-        bbo::fold_segment(n, K, f, &vb, &vs);
-        const double n_tr = n - vs, B = std::min<double>(q.batch_size, n_tr);
-        const double P = (double)d * q.hidden + q.hidden + (double)q.hidden * C + C;
-        const double steps = (double)q.epochs * std::ceil(n_tr / B);
-        cost[(size_t)c * K + f] = {(double)q.epochs * n_tr * (4.0 * d * q.hidden + 6.0 * q.hidden * C) + steps * 14.0 * P,
-                                   c * K + f};
-      }
-    }
-    std::stable_sort(cost.begin(), cost.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
-    for (int i = 0; i < n_fits; ++i) fits[i] = make_int2(cost[i].second / K, cost[i].second % K);
-  }
-  if (cudaMemcpyAsync(dcfg, configs, sizeof(bbo_mlp_config) * (size_t)n_configs, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(dfits, fits.data(), sizeof(int2) * (size_t)n_fits, cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return BBO_ERR_CUDA;
-
+  const int dp = bbo::round_up(d, 4);
   const float* Xk = X;
-  if (plan.dp != d || (reinterpret_cast<uintptr_t>(X) & 15u) != 0) {
-    const size_t total = (size_t)n * plan.dp;
-    bbo::pad_rows_kernel<<<(int)std::min<size_t>(1024, (total + 255) / 256), 256, 0, s>>>(X, n, d, plan.dp, xpad);
+  if (dp != d || (reinterpret_cast<uintptr_t>(X) & 15u) != 0) {
+    const size_t total = (size_t)n * dp;
+    bbo::pad_rows_kernel<<<(int)std::min<size_t>(1024, (total + 255) / 256), 256, 0, s>>>(X, n, d, dp, xpad);
     if (cudaGetLastError() != cudaSuccess) return BBO_ERR_CUDA;
     Xk = xpad;
   }
   if (launch_fold_permutation(n, seed, pi, s) != cudaSuccess) return BBO_ERR_CUDA;
-
-  bbo::FitArgs a{};
-  a.X = Xk; a.y = y; a.pi = pi; a.configs = dcfg; a.fits = dfits;
-  a.fold_scores = fold_scores; a.trace = nullptr; a.keep_theta = nullptr; a.queue = misc;
-  a.n_fits = n_fits; a.n_configs = n_configs;
-  a.n = n; a.d = d; a.dp = plan.dp; a.C = C; a.CS = plan.CS; a.K = K; a.task = task;
-  a.TB = plan.TB; a.trace_steps = 0; a.loss_cap = plan.loss_cap;
-  a.order_bytes = plan.order_bytes; a.seed = seed;
-  if (launch_fit_any(C, a, sd.sm_count, plan.NT, plan.smem, s) != cudaSuccess) return BBO_ERR_CUDA;
+  LaunchEnv env;  // no side streams: creating them would be a resource allocation
+  env.smem_optin = sd.smem_optin;
+  env.main = s;
+  FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr};
+  int launches = 0;
+  cudaError_t cuda_err = cudaSuccess;
+  rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, &launches, &cuda_err);
+  if (rc != BBO_OK) return rc;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(fold_scores, n_configs, K, out_scores);
   if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return BBO_ERR_CUDA;
   return BBO_OK;

@@ -1,0 +1,131 @@
+// Shared definitions of the fit kernels: argument block, shared-memory layout, k-fold
+// segments and the in-kernel permutation (sort of Philox keys).  Paper sec. 2 (cross-validation
+// score as the evaluated function); the split and shuffling rules are this library's readings.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "device_math.cuh"
+
+namespace bbo {
+
+struct Config {  // mirrors bbo_mlp_config (32 bytes)
+  int32_t hidden, batch_size, epochs;
+  float alpha, lr, beta1, beta2, eps;
+};
+
+struct FitArgs {
+  const float* X;        // [n][dp], rows 16-byte aligned
+  const float* y;        // [n]
+  const int32_t* pi;     // [n] fold permutation
+  const Config* configs; // [n_configs]
+  const int2* fits;      // this launch's (configuration, fold) list, costliest first
+  float* fold_scores;    // [n_configs * K]
+  float* trace;          // [n_configs * K * trace_steps] or null
+  float* keep_theta;     // parameters of fit (n_configs-1, K-1) in dense layout, or null
+  int32_t n_fits, n_configs;
+  int32_t n, d, dp, C, CS, K, task;
+  int32_t Hs;            // padded hidden width shared by every fit of this launch
+  int32_t TB;            // rows per sub-tile (multiple of 4, at most 32)
+  int32_t trace_steps, loss_cap;  // loss_cap: rows of the per-row loss buffer
+  int32_t order_bytes;   // bytes reserved for the epoch order (uint16 per training row)
+  uint64_t seed;
+};
+
+__host__ __device__ inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// Shared-memory layout of one fit (float offsets inside a parameter-sized block).
+struct Layout {
+  int Hs, oW1, ob1, oW2, ob2, PS, PT;
+  __host__ __device__ Layout(int d, int Hs_, int CS) {
+    Hs = Hs_;
+    oW1 = 0;
+    ob1 = d * Hs;
+    oW2 = ob1 + Hs;
+    ob2 = oW2 + Hs * CS;   // W2 has Hs rows; rows H..Hs-1 stay zero
+    PS = ob2 + CS;
+    PT = PS - ob1;         // everything but W1
+  }
+};
+
+__host__ __device__ inline int next_pow2(int x) {
+  int p = 4;
+  while (p < x) p <<= 1;
+  return p;
+}
+
+// Dynamic shared memory of one fit.  vreg: second moments of W1 live in registers.
+__host__ __device__ inline size_t fit_smem_bytes(int d, int dp, int Hs, int CS, int TB, int order_bytes,
+                                                 int loss_cap, int n_sort, bool vreg) {
+  const Layout L(d, Hs, CS);
+  size_t bytes = 4u * (size_t)(2 * L.PS + (vreg ? L.PT : L.PS));
+  bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + 8u * TB + 4u * (size_t)TB * CS;
+  const size_t xa = 8u * (size_t)TB * dp + 4u * (size_t)TB * Hs;
+  const size_t keys = 8u * (size_t)next_pow2(n_sort);
+  return bytes + (xa > keys ? xa : keys);
+}
+
+__host__ __device__ inline void fold_segment(int n, int K, int f, int* begin, int* size) {
+  const int base = n / K, rem = n % K;
+  *begin = f * base + (f < rem ? f : rem);
+  *size = base + (f < rem ? 1 : 0);
+}
+
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+  const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gmem_src) {
+  const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
+
+// Ascending bitonic sort of np2 (power of two) 64-bit keys in shared memory.
+__device__ inline void bitonic_sort(uint64_t* keys, int np2, int tid, int nt) {
+  for (int k = 2; k <= np2; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int t = tid; t < (np2 >> 1); t += nt) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int l = i | j;
+        const bool up = (i & k) == 0;
+        const uint64_t a = keys[i], b = keys[l];
+        if ((a > b) == up) { keys[i] = b; keys[l] = a; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// Permutation of 0..N-1 by ascending (random word << 32 | index); result left in the low
+// words of keys[0..N).  Leaves the block synchronised.
+__device__ inline void sorted_keys(uint64_t* keys, int N, uint64_t seed, uint32_t stream, uint32_t a,
+                                   uint32_t b, uint32_t c, int tid, int nt) {
+  const int np2 = next_pow2(N);
+  for (int blk = tid; blk < (np2 >> 2); blk += nt) {
+    const uint4 r = philox4x32_10(seed, stream, a, b, c, (uint32_t)blk);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const int i = 4 * blk + w;
+      keys[i] = i < N ? ((uint64_t)word_of(r, w) << 32) | (uint32_t)i : ~0ull;
+    }
+  }
+  __syncthreads();
+  bitonic_sort(keys, np2, tid, nt);
+}
+
+// Dataset row visited i-th in epoch `epoch`: the epoch permutation applied to the training
+// list (fold permutation with the held-out segment removed, order kept).
+__device__ inline void build_epoch_order(uint64_t* keys, uint16_t* order, const int32_t* pi, int n_tr,
+                                         int vb, int vs, uint64_t seed, uint32_t config, uint32_t fold,
+                                         uint32_t epoch, int tid, int nt) {
+  sorted_keys(keys, n_tr, seed, kStreamPerm, config, fold, epoch, tid, nt);
+  for (int i = tid; i < n_tr; i += nt) {
+    const int s = (int)(uint32_t)keys[i];
+    order[i] = (uint16_t)pi[s < vb ? s : s + vs];
+  }
+  __syncthreads();
+}
+
+}  // namespace bbo
