@@ -146,7 +146,7 @@ int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* total_ms, float* fit_ms, int32_
  * BBO_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
  * library holds those bytes until the process exits, used or not.  Hence the limits, checked
  * before anything is enqueued and reported as BBO_ERR_TOO_LARGE:
- *     n <= BBO_STATIC_MAX_ROWS,  n * roundup4(d) <= BBO_STATIC_MAX_X_FLOATS,
+ *     n <= BBO_STATIC_MAX_ROWS,  n * roundup8(d) <= BBO_STATIC_MAX_X_FLOATS,
  *     n_configs <= BBO_STATIC_MAX_CONFIGS,  n_configs * n_folds <= BBO_STATIC_MAX_FITS.
  * Shapes above the kernel caps are BBO_ERR_UNSUPPORTED as in bbo_mlp_cv_eval.
  *

@@ -18,6 +18,7 @@ LIB = os.path.join(HERE, "libbbo_mlp_cv.so")
 HEADERS = ["fit_kernel.cuh", "fit_common.cuh", "aux_kernels.cuh", "device_math.cuh", "fit_launch.h",
            os.path.join("..", "..", "include", "bbo_mlp_cv.h")]
 CLASS_COUNTS = list(range(1, 17))
+FAST_WIDTHS = list(range(56, 201, 8))   # padded hidden widths with compile-time strides
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
@@ -37,12 +38,13 @@ def _nvcc() -> str:
 
 def _units():
     units = [("bbo_mlp_cv.cu", [], "bbo_mlp_cv.o"), ("fit_dispatch.cu", [], "fit_dispatch.o")]
+    units += [("fit_fast.cu", [f"-DBBO_HSC={h}"], f"fit_fast_{h}.o") for h in reversed(FAST_WIDTHS)]
     units += [("fit_inst.cu", [f"-DBBO_CT={c}"], f"fit_inst_{c}.o") for c in CLASS_COUNTS]
     return units
 
 
 def _deps():
-    srcs = ["bbo_mlp_cv.cu", "fit_dispatch.cu", "fit_inst.cu"] + HEADERS
+    srcs = ["bbo_mlp_cv.cu", "fit_dispatch.cu", "fit_inst.cu", "fit_fast.cu"] + HEADERS
     return [os.path.join(CSRC, s) for s in srcs] + [os.path.abspath(__file__)]
 
 

@@ -21,8 +21,7 @@ static_assert(sizeof(bbo::Config) == sizeof(bbo_mlp_config), "device mirror of b
 namespace {
 
 using bbo::kMaxClasses;
-constexpr int kAuxStreams = 4;  // buckets of different hidden width overlap on these
-constexpr int kMaxThreads = 512;
+constexpr int kAuxStreams = 32;  // buckets of different hidden width overlap on these
 constexpr int kMaxRows = 16384;  // fold permutation sorts in one CTA's shared memory
 
 template <typename T>
@@ -108,46 +107,65 @@ struct Plan {
   int C, CS, dp, Hs, TB, NT, order_bytes, loss_cap, n_sort, per_sm;
   bool vreg;
   size_t smem;
+  const void* kernel;
 };
 
-// CTAs of `threads` threads and `smem` bytes that fit on one SM (registers: the kernels are
-// compiled for at most 128 per thread; warps are placed four at a time).
-int ctas_per_sm(int smem_total, int threads, size_t smem) {
-  const int by_smem = (int)((size_t)smem_total / (smem + 1024));
-  const int by_threads = 2048 / threads;
-  const int by_regs = 512 / bbo::round_up(threads, 128) ;
-  return std::max(0, std::min(by_smem, std::min(by_threads, by_regs)));
+// Resident CTAs per SM of a fit kernel instance (0 if it cannot launch).
+int kernel_occupancy(const void* kernel, int threads, size_t smem) {
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+      cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return per_sm;
 }
 
-// Plans the launch of fits of padded width Hs.  Threads: one per gradient tile of W1 (4 rows x
-// 8 columns) and two per hidden unit.  Sub-tile height: the largest of 32, 16, 8, 4 that fits.
+// Plans the launch of fits of padded width Hs.  Threads: one per gradient tile of W1 (8 rows x
+// 8 columns) and one per hidden unit.  Sub-tile height: the largest of 32, 16, 8 that fits.
 // The second moments of W1 move to registers when that lets more CTAs share an SM.
-int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bool tracing, Plan* out) {
+// probe_only: skip the occupancy queries (no CUDA calls), used by the caps query.
+int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bool tracing, bool probe_only,
+                Plan* out) {
   Plan p{};
   p.C = C;
   p.CS = bbo::round_up(C, 4);
-  p.dp = bbo::round_up(d, 4);
+  p.dp = bbo::round_up(d, 8);
   p.Hs = Hs;
   const int n_tr_max = n - n / K;
   p.order_bytes = bbo::round_up(2 * n_tr_max, 16);
   p.loss_cap = tracing ? std::min(maxB, n_tr_max) : 0;
   p.n_sort = n_tr_max;
-  const int tiles = (p.dp / 4) * (Hs / 8);
-  p.NT = bbo::round_up(std::max(std::max(tiles, 2 * Hs), 64), 32);
-  if (p.NT > kMaxThreads) return BBO_ERR_UNSUPPORTED;
+  const int tiles = (p.dp / 8) * (Hs / 8);
+  p.NT = bbo::round_up(std::max(std::max(tiles, Hs), 32), 32);
+  if (p.NT > bbo::kMaxFitThreads) return BBO_ERR_UNSUPPORTED;
   const size_t budget = (size_t)smem_optin - 256;  // static block scalars
-  const int smem_sm = smem_optin + 1024;
-  for (int TB = 32; TB >= 4; TB >>= 1) {
+  for (int TB = 32; TB >= 8; TB >>= 1) {
     const size_t plain = bbo::fit_smem_bytes(d, p.dp, Hs, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, false);
     const size_t lean = bbo::fit_smem_bytes(d, p.dp, Hs, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
     if (lean > budget) continue;
-    const int occ_plain = plain <= budget ? ctas_per_sm(smem_sm, p.NT, plain) : 0;
-    const int occ_lean = ctas_per_sm(smem_sm, p.NT, lean);
     p.TB = TB;
-    p.vreg = occ_lean > occ_plain && p.NT <= 256;
-    if (!p.vreg && plain > budget) continue;
+    if (probe_only) {
+      p.vreg = plain > budget;
+      p.smem = p.vreg ? lean : plain;
+      p.per_sm = 1;
+      *out = p;
+      return BBO_OK;
+    }
+    const void* k_plain = bbo::fit_kernel_for(C, Hs, p.dp, false);
+    const void* k_lean = bbo::fit_kernel_for(C, Hs, p.dp, true);
+    if (!k_plain || !k_lean) return BBO_ERR_UNSUPPORTED;
+    const int occ_plain = plain <= budget ? kernel_occupancy(k_plain, p.NT, plain) : 0;
+    const int occ_lean = kernel_occupancy(k_lean, p.NT, lean);
+    if (occ_plain < 1 && occ_lean < 1) continue;
+    p.vreg = occ_lean > occ_plain;
     p.smem = p.vreg ? lean : plain;
-    p.per_sm = std::max(1, p.vreg ? occ_lean : occ_plain);
+    p.per_sm = p.vreg ? occ_lean : occ_plain;
+    p.kernel = p.vreg ? k_lean : k_plain;
     *out = p;
     return BBO_OK;
   }
@@ -208,7 +226,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     int j = i;
     while (j < n_fits && items[j].Hs == items[i].Hs) ++j;
     Group g{i, j - i, {}};
-    const int rc = plan_bucket(env.smem_optin, n, d, C, K, items[i].Hs, maxB, trace_steps > 0, &g.plan);
+    const int rc = plan_bucket(env.smem_optin, n, d, C, K, items[i].Hs, maxB, trace_steps > 0, false, &g.plan);
     if (rc != BBO_OK) return rc;
     groups.push_back(g);
     i = j;
@@ -235,7 +253,10 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     a.Hs = g.plan.Hs; a.TB = g.plan.TB; a.trace_steps = trace_steps; a.loss_cap = g.plan.loss_cap;
     a.order_bytes = g.plan.order_bytes; a.seed = seed;
     cudaStream_t s = side ? env.aux[gi % env.n_aux] : env.main;
-    if ((e = bbo::launch_fit(C, a, g.plan.vreg, g.plan.NT, g.count, g.plan.smem, s)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
+    void* kargs[] = {&a};
+    // groups of different width may share one kernel instance: its limit is per launch
+    if ((e = cudaFuncSetAttribute(g.plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.plan.smem)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
+    if ((e = cudaLaunchKernel(g.plan.kernel, dim3(g.count), dim3(g.plan.NT), kargs, g.plan.smem, s)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
     ++*launches;
   }
   if (side) {
@@ -376,7 +397,7 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   }
 
   const bool tracing = h->opt.trace_steps > 0;
-  const int dp = bbo::round_up(d, 4);
+  const int dp = bbo::round_up(d, 8);
   const int n_fits = n_configs * K;
   BBO_CUDA(h, h->configs.reserve(n_configs));
   BBO_CUDA(h, h->fits.reserve(n_fits));
@@ -532,7 +553,7 @@ int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* 
   // widest hidden layer for (d, C) on a 1797-row, 5-fold problem with the smallest sub-tile
   auto fits_H = [&](int dd, int H) {
     Plan p;
-    return plan_bucket(h->smem_optin, 1797, dd, n_classes, 5, bbo::round_up(H, 8), 1, false, &p) == BBO_OK;
+    return plan_bucket(h->smem_optin, 1797, dd, n_classes, 5, bbo::round_up(H, 8), 1, false, true, &p) == BBO_OK;
   };
   if (max_hidden) {
     int lo = 0, hi = 4096;
@@ -630,7 +651,7 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
   if (n64 < 2 || d < 1 || K < 2 || K > n64 || n_configs < 1 || n_classes < 0 || n_classes > kMaxClasses)
     return BBO_ERR_INVALID_ARG;
   if (task != BBO_TASK_CLASSIFICATION && task != BBO_TASK_REGRESSION) return BBO_ERR_INVALID_ARG;
-  const int64_t dp64 = (int64_t)(d + 3) / 4 * 4;
+  const int64_t dp64 = (int64_t)(d + 7) / 8 * 8;
   if (n64 > BBO_STATIC_MAX_ROWS || n64 * dp64 > BBO_STATIC_MAX_X_FLOATS || n_configs > BBO_STATIC_MAX_CONFIGS ||
       (int64_t)n_configs * K > BBO_STATIC_MAX_FITS)
     return BBO_ERR_TOO_LARGE;
@@ -677,7 +698,7 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
     if (C > kMaxClasses) return BBO_ERR_UNSUPPORTED;
   }
 
-  const int dp = bbo::round_up(d, 4);
+  const int dp = bbo::round_up(d, 8);
   const float* Xk = X;
   if (dp != d || (reinterpret_cast<uintptr_t>(X) & 15u) != 0) {
     const size_t total = (size_t)n * dp;

@@ -1,0 +1,19 @@
+// Instantiates the compile-time-stride fit kernels (64 padded features, 10 classes) for one
+// padded hidden width (BBO_HSC).
+#include "fit_kernel.cuh"
+#include "fit_launch.h"
+
+#ifndef BBO_HSC
+#error "compile with -DBBO_HSC=<padded hidden width>"
+#endif
+
+namespace bbo {
+
+template <>
+const void* fast_fit_kernel<BBO_HSC>(bool vreg) {
+  constexpr int NT = (BBO_HSC + 31) / 32 * 32;
+  if (vreg) return reinterpret_cast<const void*>(&mlp_cv_fit_kernel<kFastClasses, true, BBO_HSC, kFastDp, NT, 1>);
+  return reinterpret_cast<const void*>(&mlp_cv_fit_kernel<kFastClasses, false, BBO_HSC, kFastDp, NT, 1>);
+}
+
+}  // namespace bbo

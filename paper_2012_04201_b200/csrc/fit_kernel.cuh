@@ -12,16 +12,19 @@
 // once per step.  Threads own outputs, never partial sums: there is no split reduction
 // anywhere on the training path.
 //
-// Work decomposition per minibatch, in sub-tiles of TB rows (H padded to Hs = 8*ceil(H/8)):
+// Work decomposition per minibatch, in sub-tiles of TB rows (H padded to Hs = 8*ceil(H/8),
+// d padded to dp = 8*ceil(d/8)); about Hs threads per fit, few and register-heavy, because
+// shared-memory instruction issue, not capacity, is what limits the register-tiled loops:
 //   stage   cp.async gather of the next sub-tile's rows, double buffered
-//   hidden  4x4 register tiles of A1 = relu(X W1 + b1), k ascending
-//   output  one lane per z2[b][o] (32/C rows per warp), j ascending, softmax and loss
-//           derivative with warp shuffles in the same lanes
-//   gW2     two threads per hidden unit, each half of the classes, b ascending, in registers
-//   delta1  4x4 register tiles (columns strided by Hs/4), o ascending, in place over A1
-//   gW1     4x8 register tiles that persist across sub-tiles, b ascending; the owner applies
+//   hidden  8x4 register tiles of A1 = relu(X W1 + b1), k ascending
+//   output  one lane per z2[b][o] (32/C rows per warp, two rows in flight per lane),
+//           j ascending, softmax and loss derivative with warp shuffles in the same lanes
+//   unit    one thread per hidden unit j: gW2[j][:], delta1[:, j] (in place over A1), gb1[j]
+//   gW1     8x8 register tiles that persist across sub-tiles, b ascending; the owner applies
 //           the L2 term and Adam to exactly its elements (second moments of W1 may stay in
 //           the owner's registers for the whole fit)
+// HSC / DPC: compile-time Hs / dp (0 = taken from the arguments) so that every shared-memory
+// access of the hot loops is base + immediate.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -41,45 +44,49 @@ struct FitView {  // per-fit pointers into shared memory
 // Asynchronous gather of nb dataset rows into buffer `buf` of Xs / ys.  Rows nb..TB-1 are
 // zero-filled so that the forward tiles read defined values.  row_of(r) = dataset row.
 template <typename RowFn>
-__device__ __forceinline__ void stage_rows_async(const FitArgs& a, const FitView& v, int buf, int nb,
+__device__ __forceinline__ void stage_rows_async(const FitArgs& a, const FitView& v, int dp, int buf, int nb,
                                                  RowFn row_of, int tid, int nt) {
-  const int vec = a.dp >> 2;
-  float* xs = v.Xs + buf * a.TB * a.dp;
+  const int vec = dp >> 2;
+  float* xs = v.Xs + buf * a.TB * dp;
   for (int i = tid; i < a.TB * vec; i += nt) {
     const int r = i / vec, q = i - r * vec;
     float4* dst = reinterpret_cast<float4*>(xs) + i;
-    if (r < nb) cp_async_16(dst, reinterpret_cast<const float4*>(a.X + (size_t)row_of(r) * a.dp) + q);
+    if (r < nb) cp_async_16(dst, reinterpret_cast<const float4*>(a.X + (size_t)row_of(r) * dp) + q);
     else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   for (int r = tid; r < nb; r += nt) cp_async_4(v.ys + buf * a.TB + r, a.y + row_of(r));
   cp_async_commit();
 }
 
-// A1 = relu(Xs W1 + b1) for the TB-row tile; each thread owns 4x4 outputs, k ascending.
-__device__ __forceinline__ void forward_hidden(const FitArgs& a, const FitView& v, const Layout& L,
-                                               const float* xs, int nb, int tid, int nt) {
-  const int JG = L.Hs >> 2, n_tiles = ((nb + 3) >> 2) * JG;
-  const float* W1 = v.W + L.oW1;
-  const int d4 = a.d >> 2, dp = a.dp, Hs = L.Hs;
+__device__ __forceinline__ float f4_get(const float4& v, int i) {
+  return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
+}
+
+// A1 = relu(Xs W1 + b1) for the sub-tile; each thread owns 8 rows x 4 columns, k ascending.
+__device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L, const float* xs, int d, int dp,
+                                               int Hs, int nb, int tid, int nt) {
+  const int JG = Hs >> 2, n_tiles = ((nb + 7) >> 3) * JG;
+  const int d4 = d >> 2;
   for (int t = tid; t < n_tiles; t += nt) {
     const int bg = t / JG, jg = t - bg * JG;
-    const int b0 = bg << 2, j0 = jg << 2;
+    const int b0 = bg << 3, j0 = jg << 2;
     const float4 bias = *reinterpret_cast<const float4*>(v.W + L.ob1 + j0);
-    float acc[4][4];
+    float acc[8][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) { acc[i][0] = bias.x; acc[i][1] = bias.y; acc[i][2] = bias.z; acc[i][3] = bias.w; }
+    for (int i = 0; i < 8; ++i) { acc[i][0] = bias.x; acc[i][1] = bias.y; acc[i][2] = bias.z; acc[i][3] = bias.w; }
     const float* xrow = xs + b0 * dp;
-    const float* wp = W1 + j0;
+    const float* wp = v.W + L.oW1 + j0;
+#pragma unroll 2
     for (int k4 = 0; k4 < d4; ++k4) {
-      float4 xv[4];
+      float4 xv[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) xv[i] = *reinterpret_cast<const float4*>(xrow + i * dp + 4 * k4);
+      for (int i = 0; i < 8; ++i) xv[i] = *reinterpret_cast<const float4*>(xrow + i * dp + 4 * k4);
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
         const float4 w = *reinterpret_cast<const float4*>(wp + (4 * k4 + kk) * Hs);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float x = kk == 0 ? xv[i].x : (kk == 1 ? xv[i].y : (kk == 2 ? xv[i].z : xv[i].w));
+        for (int i = 0; i < 8; ++i) {
+          const float x = f4_get(xv[i], kk);
           acc[i][0] = __fmaf_rn(x, w.x, acc[i][0]);
           acc[i][1] = __fmaf_rn(x, w.y, acc[i][1]);
           acc[i][2] = __fmaf_rn(x, w.z, acc[i][2]);
@@ -87,10 +94,10 @@ __device__ __forceinline__ void forward_hidden(const FitArgs& a, const FitView& 
         }
       }
     }
-    for (int k = d4 << 2; k < a.d; ++k) {
+    for (int k = d4 << 2; k < d; ++k) {
       const float4 w = *reinterpret_cast<const float4*>(wp + k * Hs);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < 8; ++i) {
         const float x = xrow[i * dp + k];
         acc[i][0] = __fmaf_rn(x, w.x, acc[i][0]);
         acc[i][1] = __fmaf_rn(x, w.y, acc[i][1]);
@@ -99,7 +106,7 @@ __device__ __forceinline__ void forward_hidden(const FitArgs& a, const FitView& 
       }
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 8; ++i) {
       float4 o;
       o.x = acc[i][0] > 0.f ? acc[i][0] : 0.f;
       o.y = acc[i][1] > 0.f ? acc[i][1] : 0.f;
@@ -110,25 +117,35 @@ __device__ __forceinline__ void forward_hidden(const FitArgs& a, const FitView& 
   }
 }
 
-// z2[b][o] = b2[o] + sum_j A1[b][j] W2[j][o], j ascending, for lane (r, o) of a warp that
-// holds 32/CT rows.  Returns the lane's logit (undefined for inactive lanes).
-template <int CT>
-__device__ __forceinline__ float output_logit(const FitView& v, const Layout& L, int CS, int H, int b, int o,
-                                              bool active) {
-  if (!active) return 0.f;
-  float acc = v.W[L.ob2 + o];
-  const float* arow = v.A1 + b * L.Hs;
+// Logits of up to two rows per lane: z2[b][o] = b2[o] + sum_j A1[b][j] W2[j][o], j ascending.
+// Row b0 is valid when act0, row b1 when act1 (act1 implies act0).
+__device__ __forceinline__ void output_logits2(const FitView& v, const Layout& L, int CS, int Hs, int H, int o,
+                                               int b0, bool act0, int b1, bool act1, float& z0, float& z1) {
+  z0 = 0.f;
+  z1 = 0.f;
+  if (!act0) return;
+  const float bias = v.W[L.ob2 + o];
+  float acc0 = bias, acc1 = bias;
+  const float* r0 = v.A1 + b0 * Hs;
+  const float* r1 = v.A1 + (act1 ? b1 : b0) * Hs;
   const float* wcol = v.W + L.oW2 + o;
   int j = 0;
-  for (; j + 8 <= H; j += 8) {
-    float av[8], wv[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) { av[u] = arow[j + u]; wv[u] = wcol[(j + u) * CS]; }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) acc = __fmaf_rn(av[u], wv[u], acc);
+  for (; j + 4 <= H; j += 4) {
+    const float4 a0 = *reinterpret_cast<const float4*>(r0 + j);
+    const float4 a1 = *reinterpret_cast<const float4*>(r1 + j);
+    const float w0 = wcol[j * CS], w1 = wcol[(j + 1) * CS], w2 = wcol[(j + 2) * CS], w3 = wcol[(j + 3) * CS];
+    acc0 = __fmaf_rn(a0.x, w0, acc0); acc1 = __fmaf_rn(a1.x, w0, acc1);
+    acc0 = __fmaf_rn(a0.y, w1, acc0); acc1 = __fmaf_rn(a1.y, w1, acc1);
+    acc0 = __fmaf_rn(a0.z, w2, acc0); acc1 = __fmaf_rn(a1.z, w2, acc1);
+    acc0 = __fmaf_rn(a0.w, w3, acc0); acc1 = __fmaf_rn(a1.w, w3, acc1);
   }
-  for (; j < H; ++j) acc = __fmaf_rn(arow[j], wcol[j * CS], acc);
-  return acc;
+  for (; j < H; ++j) {
+    const float w = wcol[j * CS];
+    acc0 = __fmaf_rn(r0[j], w, acc0);
+    acc1 = __fmaf_rn(r1[j], w, acc1);
+  }
+  z0 = acc0;
+  z1 = acc1;
 }
 
 // Adam on one parameter with its gradient (L2 term already added for weights).
@@ -146,18 +163,44 @@ struct BlockShared {  // block-wide scalars
   float red[32];
 };
 
-// The whole fit.  CT: class count (compile time).  VR: second moments of W1 in registers.
-template <int CT, bool VR>
+// Softmax (or residual) of one row held across CT lanes starting at lane `obase`; returns this
+// lane's loss derivative.  All 32 lanes must call it.
+template <int CT>
+__device__ __forceinline__ float row_delta(const FitView& v, int task, float z, float yv, int ocol, int obase,
+                                           bool active, float invB, bool want_loss, int loss_idx) {
+  if (task == 0) {
+    const int label = (int)yv;
+    float mx = __shfl_sync(0xffffffffu, z, obase);
+#pragma unroll
+    for (int o = 1; o < CT; ++o) { const float t = __shfl_sync(0xffffffffu, z, obase + o); if (t > mx) mx = t; }
+    const float ex = spec_expf(__fsub_rn(z, mx));
+    float sum = 0.f;
+#pragma unroll
+    for (int o = 0; o < CT; ++o) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, ex, obase + o));
+    const float pr = __fdiv_rn(ex, sum);
+    if (want_loss) {
+      const float zl = __shfl_sync(0xffffffffu, z, obase + (active ? label : 0));
+      if (active && ocol == 0) v.lossb[loss_idx] = __fsub_rn(logf(sum), __fsub_rn(zl, mx));
+    }
+    return __fmul_rn(__fsub_rn(pr, ocol == label ? 1.0f : 0.0f), invB);
+  }
+  const float r = __fsub_rn(z, yv);
+  if (want_loss && active) v.lossb[loss_idx] = __fmul_rn(__fmul_rn(0.5f, r), r);
+  return __fmul_rn(r, invB);
+}
+
+// The whole fit.  CT: class count.  VR: second moments of W1 in registers.
+template <int CT, bool VR, int HSC, int DPC>
 __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, BlockShared& sh) {
   constexpr int RW = 32 / CT;           // rows per warp in the output phase
-  constexpr int CA = (CT + 1) / 2;      // classes per thread in the gW2 phase
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
   const int2 cf = a.fits[q];
   const int config = cf.x, fold = cf.y;
   const Config c = a.configs[config];
-  const int H = c.hidden, d = a.d, dp = a.dp, CS = a.CS, TB = a.TB;
-  const Layout L(d, a.Hs, CS);
-  const int Hs = L.Hs;
+  const int H = c.hidden, d = a.d, CS = a.CS, TB = a.TB;
+  const int dp = DPC ? DPC : a.dp;
+  const int Hs = HSC ? HSC : a.Hs;
+  const Layout L(d, Hs, CS);
   int vb, vs;
   fold_segment(a.n, a.K, fold, &vb, &vs);
   const int n_tr = a.n - vs;
@@ -216,36 +259,32 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   __syncthreads();
 
   // ---- thread roles ----
-  const int KG = dp >> 2, JG8 = Hs >> 3, JG4 = Hs >> 2;
+  const int KG = dp >> 3, JG8 = Hs >> 3;
   const bool has_tile = tid < KG * JG8;            // gW1 tile owner (host guarantees KG*JG8 <= nt)
   const int kg = has_tile ? tid / JG8 : 0, jg = has_tile ? tid - kg * JG8 : 0;
-  const int k0 = kg << 2, jA = jg << 2, jB = (jg + JG8) << 2;
-  const bool bias_owner = has_tile && kg == 0;     // also owns gb1 of its eight columns
-  const int hj = tid >> 1, part = tid & 1;          // gW2: hidden unit and class half
-  const bool w2_role = hj < H && (CT > 1 || part == 0);
-  const int oa = part * CA;                         // first class of this thread's half
-  const bool o_role = tid < CT;                     // gb2 owner
-  // output phase: lane (r, o)
+  const int k0 = kg << 3, jA = jg << 2, jB = (jg + JG8) << 2;
+  const bool unit_role = tid < H;                   // hidden unit tid: W2 row, b1, delta1 column
+  const bool o_role = tid < CT;                     // gb2 / b2 owner
   const int orow = lane / CT, ocol = lane - orow * CT, obase = orow < RW ? orow * CT : 0;
+  const int rows_per_pass = n_warps * RW;
 
   const float beta1 = c.beta1, beta2 = c.beta2, eps = c.eps;
   const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
   double p1 = 1.0, p2 = 1.0;  // running beta^t (thread 0 only)
   int step_no = 0;
-  float v1[4][8];             // second moments of this thread's W1 tile (VR only)
+  float v1[8][8];             // second moments of this thread's W1 tile (VR only)
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 8; ++i)
 #pragma unroll
     for (int j = 0; j < 8; ++j) v1[i][j] = 0.f;
 
   for (int e = 0; e < c.epochs; ++e) {
     build_epoch_order(v.keys, v.order, a.pi, n_tr, vb, vs, a.seed, config, fold, e, tid, nt);
-    // first sub-tile of the epoch
     int buf = 0;
-    {
+    {  // first sub-tile of the epoch
       const int Bs0 = n_tr < B ? n_tr : B, nb0 = Bs0 < TB ? Bs0 : TB;
       const uint16_t* rows = v.order;
-      stage_rows_async(a, v, 0, nb0, [&](int r) { return (int)rows[r]; }, tid, nt);
+      stage_rows_async(a, v, dp, 0, nb0, [&](int r) { return (int)rows[r]; }, tid, nt);
     }
     for (int s0 = 0; s0 < n_tr; s0 += B) {
       const int Bs = (n_tr - s0) < B ? (n_tr - s0) : B;
@@ -257,16 +296,14 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         p2 *= (double)beta2;
         sh.step[step_no & 1] = (float)((double)c.lr * sqrt(1.0 - p2) / (1.0 - p1));
       }
-      float g1[4][8];
+      float g1[8][8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 8; ++i)
 #pragma unroll
         for (int j = 0; j < 8; ++j) g1[i][j] = 0.f;
-      float g2[CA], gb1[8], gb2 = 0.f;
+      float g2[CT], w2[CT], gb1 = 0.f, gb2 = 0.f;
 #pragma unroll
-      for (int o = 0; o < CA; ++o) g2[o] = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) gb1[j] = 0.f;
+      for (int o = 0; o < CT; ++o) { g2[o] = 0.f; w2[o] = unit_role ? v.W[L.oW2 + tid * CS + o] : 0.f; }
 
       for (int t0 = 0; t0 < Bs; t0 += TB) {
         const int nb = (Bs - t0) < TB ? (Bs - t0) : TB;
@@ -281,121 +318,70 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           if (ns0 < n_tr) {
             const int nnb = (nBs - nt0) < TB ? (nBs - nt0) : TB;
             const uint16_t* rows = v.order + ns0 + nt0;
-            stage_rows_async(a, v, buf ^ 1, nnb, [&](int r) { return (int)rows[r]; }, tid, nt);
+            stage_rows_async(a, v, dp, buf ^ 1, nnb, [&](int r) { return (int)rows[r]; }, tid, nt);
           }
         }
-        forward_hidden(a, v, L, xs, nb, tid, nt);
+        forward_hidden(v, L, xs, d, dp, Hs, nb, tid, nt);
         __syncthreads();
 
         // ---- output layer, softmax / residual, loss derivative (lanes own logits) ----
-        for (int bw = warp * RW; bw < nb; bw += n_warps * RW) {
-          const int b = bw + orow;
-          const bool active = orow < RW && b < nb;
-          const float z = output_logit<CT>(v, L, CS, H, b, ocol, active);
-          const float yv = active ? ysb[b] : 0.f;
-          float delta;
-          if (a.task == 0) {
-            const int label = (int)yv;
-            float mx = __shfl_sync(0xffffffffu, z, obase);
-#pragma unroll
-            for (int o = 1; o < CT; ++o) { const float t = __shfl_sync(0xffffffffu, z, obase + o); if (t > mx) mx = t; }
-            const float ex = spec_expf(__fsub_rn(z, mx));
-            float sum = 0.f;
-#pragma unroll
-            for (int o = 0; o < CT; ++o) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, ex, obase + o));
-            const float pr = __fdiv_rn(ex, sum);
-            delta = __fmul_rn(__fsub_rn(pr, ocol == label ? 1.0f : 0.0f), invB);
-            if (want_loss) {
-              const float zl = __shfl_sync(0xffffffffu, z, obase + (active ? label : 0));
-              if (active && ocol == 0) v.lossb[t0 + b] = __fsub_rn(logf(sum), __fsub_rn(zl, mx));
-            }
-          } else {
-            const float r = __fsub_rn(z, yv);
-            delta = __fmul_rn(r, invB);
-            if (want_loss && active) v.lossb[t0 + b] = __fmul_rn(__fmul_rn(0.5f, r), r);
+        for (int bw = warp * RW; bw < nb; bw += 2 * rows_per_pass) {
+          const int b0 = bw + orow, b1 = b0 + rows_per_pass;
+          const bool act0 = orow < RW && b0 < nb, act1 = orow < RW && b1 < nb;
+          float z0, z1;
+          output_logits2(v, L, CS, Hs, H, ocol, b0, act0, b1, act1, z0, z1);
+          const float d0 = row_delta<CT>(v, a.task, z0, act0 ? ysb[b0] : 0.f, ocol, obase, act0, invB, want_loss, t0 + b0);
+          if (act0) v.D2[b0 * CS + ocol] = d0;
+          if (bw + rows_per_pass < nb) {  // warp-uniform
+            const float d1 = row_delta<CT>(v, a.task, z1, act1 ? ysb[b1] : 0.f, ocol, obase, act1, invB, want_loss, t0 + b1);
+            if (act1) v.D2[b1 * CS + ocol] = d1;
           }
-          if (active) v.D2[b * CS + ocol] = delta;
         }
         __syncthreads();
 
-        // ---- gW2[j][oa..oa+CA) += A1[b][j] * delta2[b][o], gb2[o] += delta2[b][o]; b ascending ----
-        if (w2_role) {
-          const float* ap = v.A1 + hj;
-          const float* dp2 = v.D2 + oa;
-#pragma unroll 4
+        // ---- hidden unit tid: gW2[tid][:], delta1[:, tid] in place over A1, gb1[tid]; b ascending ----
+        if (unit_role) {
+          float* ap = v.A1 + tid;
+#pragma unroll 2
           for (int b = 0; b < nb; ++b) {
             const float a1 = ap[b * Hs];
+            float dl[(CT + 3) / 4 * 4];
 #pragma unroll
-            for (int o = 0; o < CA; ++o)
-              if (oa + o < CT) g2[o] = __fmaf_rn(a1, dp2[b * CS + o], g2[o]);
+            for (int o4 = 0; o4 < (CT + 3) / 4; ++o4) {
+              const float4 t = *reinterpret_cast<const float4*>(v.D2 + b * CS + 4 * o4);
+              dl[4 * o4] = t.x; dl[4 * o4 + 1] = t.y; dl[4 * o4 + 2] = t.z; dl[4 * o4 + 3] = t.w;
+            }
+            float acc = 0.f;
+#pragma unroll
+            for (int o = 0; o < CT; ++o) {
+              g2[o] = __fmaf_rn(a1, dl[o], g2[o]);
+              acc = __fmaf_rn(dl[o], w2[o], acc);
+            }
+            const float d1 = a1 > 0.f ? acc : 0.f;
+            ap[b * Hs] = d1;
+            gb1 = __fadd_rn(gb1, d1);
           }
         }
         if (o_role) for (int b = 0; b < nb; ++b) gb2 = __fadd_rn(gb2, v.D2[b * CS + tid]);
         __syncthreads();
 
-        // ---- delta1 = (delta2 W2^T) masked by A1 > 0, in place; 4 rows x 4 strided columns ----
-        {
-          const int n_tiles = ((nb + 3) >> 2) * JG4;
-          for (int t = tid; t < n_tiles; t += nt) {
-            const int bg = t / JG4, jl = t - bg * JG4, b0 = bg << 2;
-            float acc[4][4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-              for (int jj = 0; jj < 4; ++jj) acc[i][jj] = 0.f;
-#pragma unroll
-            for (int o4 = 0; o4 < (CT + 3) / 4; ++o4) {
-              float4 dl[4], w2[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) dl[i] = *reinterpret_cast<const float4*>(v.D2 + (b0 + i) * CS + 4 * o4);
-#pragma unroll
-              for (int jj = 0; jj < 4; ++jj) w2[jj] = *reinterpret_cast<const float4*>(v.W + L.oW2 + (jl + jj * JG4) * CS + 4 * o4);
-#pragma unroll
-              for (int oo = 0; oo < 4; ++oo) {
-                if (4 * o4 + oo < CT) {
-#pragma unroll
-                  for (int i = 0; i < 4; ++i) {
-                    const float dv = oo == 0 ? dl[i].x : (oo == 1 ? dl[i].y : (oo == 2 ? dl[i].z : dl[i].w));
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                      const float wv = oo == 0 ? w2[jj].x : (oo == 1 ? w2[jj].y : (oo == 2 ? w2[jj].z : w2[jj].w));
-                      acc[i][jj] = __fmaf_rn(dv, wv, acc[i][jj]);
-                    }
-                  }
-                }
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-              for (int jj = 0; jj < 4; ++jj) {
-                float* cell = v.A1 + (b0 + i) * Hs + jl + jj * JG4;
-                *cell = *cell > 0.f ? acc[i][jj] : 0.f;
-              }
-          }
-        }
-        __syncthreads();
-
-        // ---- gW1 tile: rows k0..k0+3, columns jA..jA+3 and jB..jB+3, b ascending; gb1 ----
+        // ---- gW1 tile: rows k0..k0+7, columns jA..jA+3 and jB..jB+3, b ascending ----
         if (has_tile) {
           const float* xp = xs + k0;
           const float* da = v.A1 + jA;
           const float* db = v.A1 + jB;
 #pragma unroll 2
           for (int b = 0; b < nb; ++b) {
-            const float4 xv = *reinterpret_cast<const float4*>(xp + b * dp);
+            const float4 x0 = *reinterpret_cast<const float4*>(xp + b * dp);
+            const float4 x1 = *reinterpret_cast<const float4*>(xp + b * dp + 4);
             const float4 dA = *reinterpret_cast<const float4*>(da + b * Hs);
             const float4 dB = *reinterpret_cast<const float4*>(db + b * Hs);
-            const float xk[4] = {xv.x, xv.y, xv.z, xv.w};
+            const float xk[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
             const float ds[8] = {dA.x, dA.y, dA.z, dA.w, dB.x, dB.y, dB.z, dB.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < 8; ++i)
 #pragma unroll
               for (int j = 0; j < 8; ++j) g1[i][j] = __fmaf_rn(xk[i], ds[j], g1[i][j]);
-            if (bias_owner) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j) gb1[j] = __fadd_rn(gb1[j], ds[j]);
-            }
           }
         }
         buf ^= 1;
@@ -426,7 +412,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       const float step = sh.step[step_no & 1];
       if (has_tile) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 8; ++i) {
           const int k = k0 + i;
           if (k < d) {
 #pragma unroll
@@ -437,11 +423,10 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
               float4 vv;
               if (VR) vv = make_float4(v1[i][4 * half], v1[i][4 * half + 1], v1[i][4 * half + 2], v1[i][4 * half + 3]);
               else vv = *reinterpret_cast<float4*>(v.V + off);
-              const float* g = &g1[i][4 * half];
-              adam_one(w.x, m.x, vv.x, __fmaf_rn(aB, w.x, g[0]), beta1, beta2, omb1, omb2, step, eps);
-              adam_one(w.y, m.y, vv.y, __fmaf_rn(aB, w.y, g[1]), beta1, beta2, omb1, omb2, step, eps);
-              adam_one(w.z, m.z, vv.z, __fmaf_rn(aB, w.z, g[2]), beta1, beta2, omb1, omb2, step, eps);
-              adam_one(w.w, m.w, vv.w, __fmaf_rn(aB, w.w, g[3]), beta1, beta2, omb1, omb2, step, eps);
+              adam_one(w.x, m.x, vv.x, __fmaf_rn(aB, w.x, g1[i][4 * half]), beta1, beta2, omb1, omb2, step, eps);
+              adam_one(w.y, m.y, vv.y, __fmaf_rn(aB, w.y, g1[i][4 * half + 1]), beta1, beta2, omb1, omb2, step, eps);
+              adam_one(w.z, m.z, vv.z, __fmaf_rn(aB, w.z, g1[i][4 * half + 2]), beta1, beta2, omb1, omb2, step, eps);
+              adam_one(w.w, m.w, vv.w, __fmaf_rn(aB, w.w, g1[i][4 * half + 3]), beta1, beta2, omb1, omb2, step, eps);
               *reinterpret_cast<float4*>(v.W + off) = w;
               *reinterpret_cast<float4*>(v.M + off) = m;
               if (VR) { v1[i][4 * half] = vv.x; v1[i][4 * half + 1] = vv.y; v1[i][4 * half + 2] = vv.z; v1[i][4 * half + 3] = vv.w; }
@@ -449,34 +434,24 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
             }
           }
         }
-        if (bias_owner) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int col = (j < 4 ? jA : jB) + (j & 3);
-            if (col < H) {
-              const int off = L.ob1 + col;
-              adam_one(v.W[off], v.M[off], v.V[off], gb1[j], beta1, beta2, omb1, omb2, step, eps);
-            }
-          }
-        }
       }
-      if (w2_role) {
+      if (unit_role) {
 #pragma unroll
-        for (int o = 0; o < CA; ++o) {
-          if (oa + o < CT) {
-            const int off = L.oW2 + hj * CS + oa + o;
-            float w = v.W[off];
-            adam_one(w, v.M[off], v.V[off], __fmaf_rn(aB, w, g2[o]), beta1, beta2, omb1, omb2, step, eps);
-            v.W[off] = w;
-          }
+        for (int o = 0; o < CT; ++o) {
+          const int off = L.oW2 + tid * CS + o;
+          float w = w2[o];
+          adam_one(w, v.M[off], v.V[off], __fmaf_rn(aB, w, g2[o]), beta1, beta2, omb1, omb2, step, eps);
+          v.W[off] = w;
         }
+        const int off = L.ob1 + tid;
+        adam_one(v.W[off], v.M[off], v.V[off], gb1, beta1, beta2, omb1, omb2, step, eps);
       }
       if (o_role) {
         const int off = L.ob2 + tid;
         adam_one(v.W[off], v.M[off], v.V[off], gb2, beta1, beta2, omb1, omb2, step, eps);
       }
       ++step_no;
-      // the barrier at the top of the next sub-tile (or of the sort) orders these writes
+      // the barrier at the top of the next sub-tile (or after the epoch) orders these writes
     }
     __syncthreads();
   }
@@ -486,26 +461,33 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   __syncthreads();
   for (int t0 = 0; t0 < vs; t0 += TB) {
     const int nb = (vs - t0) < TB ? (vs - t0) : TB;
-    stage_rows_async(a, v, 0, nb, [&](int r) { return a.pi[vb + t0 + r]; }, tid, nt);
+    stage_rows_async(a, v, dp, 0, nb, [&](int r) { return a.pi[vb + t0 + r]; }, tid, nt);
     cp_async_wait_all();
     __syncthreads();
-    forward_hidden(a, v, L, v.Xs, nb, tid, nt);
+    forward_hidden(v, L, v.Xs, d, dp, Hs, nb, tid, nt);
     __syncthreads();
-    for (int bw = warp * RW; bw < nb; bw += n_warps * RW) {
-      const int b = bw + orow;
-      const bool active = orow < RW && b < nb;
-      const float z = output_logit<CT>(v, L, CS, H, b, ocol, active);
-      if (a.task == 0) {
-        float best = __shfl_sync(0xffffffffu, z, obase);
-        int besti = 0;
+    for (int bw = warp * RW; bw < nb; bw += 2 * rows_per_pass) {
+      const int b0 = bw + orow, b1 = b0 + rows_per_pass;
+      const bool act0 = orow < RW && b0 < nb, act1 = orow < RW && b1 < nb;
+      float zz[2];
+      output_logits2(v, L, CS, Hs, H, ocol, b0, act0, b1, act1, zz[0], zz[1]);
 #pragma unroll
-        for (int o = 1; o < CT; ++o) {
-          const float t = __shfl_sync(0xffffffffu, z, obase + o);
-          if (t > best) { best = t; besti = o; }
+      for (int cidx = 0; cidx < 2; ++cidx) {
+        const float z = zz[cidx];
+        const int b = cidx ? b1 : b0;
+        const bool act = cidx ? act1 : act0;
+        if (a.task == 0) {
+          float best = __shfl_sync(0xffffffffu, z, obase);
+          int besti = 0;
+#pragma unroll
+          for (int o = 1; o < CT; ++o) {
+            const float t = __shfl_sync(0xffffffffu, z, obase + o);
+            if (t > best) { best = t; besti = o; }
+          }
+          if (act && ocol == 0 && besti == (int)v.ys[b]) atomicAdd(&sh.correct, 1);
+        } else if (act) {
+          v.D2[b * CS] = __fsub_rn(z, v.ys[b]);
         }
-        if (active && ocol == 0 && besti == (int)v.ys[b]) atomicAdd(&sh.correct, 1);
-      } else if (active) {
-        v.D2[b * CS] = __fsub_rn(z, v.ys[b]);
       }
     }
     __syncthreads();
@@ -536,11 +518,11 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 }
 
 // One CTA per fit; blockIdx.x indexes this launch's fit list (costliest first).
-template <int CT, bool VR, int NTMAX, int MINB>
+template <int CT, bool VR, int HSC, int DPC, int NTMAX, int MINB>
 __global__ void __launch_bounds__(NTMAX, MINB) mlp_cv_fit_kernel(const FitArgs a) {
   extern __shared__ __align__(16) float smem[];
   __shared__ BlockShared sh;
-  run_fit<CT, VR>(a, blockIdx.x, smem, sh);
+  run_fit<CT, VR, HSC, DPC>(a, blockIdx.x, smem, sh);
 }
 
 }  // namespace bbo

@@ -1,6 +1,7 @@
-// Host-side entry to the fit kernels.  The kernels are templates on the class count; each
-// class count is compiled in its own translation unit (fit_inst.cu with -DBBO_CT=<n>) so the
-// library builds in parallel, and this dispatcher picks the instance at run time.
+// Host-side access to the fit kernels.  The kernels are templates on the class count (and,
+// for the 64-feature / 10-class shape, on the padded hidden width); every instance is
+// compiled in its own translation unit so the library builds in parallel, and this table
+// returns the instance for a launch at run time.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -9,12 +10,17 @@
 namespace bbo {
 
 constexpr int kMaxClasses = 16;
+constexpr int kMaxFitThreads = 256;  // launch bound of every fit kernel
 
-// Launches `grid` CTAs of `threads` threads (one per fit of a.fits) with `smem` bytes of
-// dynamic shared memory.  vreg: second moments of W1 kept in registers.
-template <int CT>
-cudaError_t launch_fit_ct(const FitArgs& a, bool vreg, int threads, int grid, size_t smem, cudaStream_t s);
+// Fast-path shape: compile-time strides for dp == kFastDp, C == kFastClasses and
+// Hs in [kFastHsMin, kFastHsMax] (multiples of 8).
+constexpr int kFastDp = 64, kFastClasses = 10, kFastHsMin = 56, kFastHsMax = 200;
 
-cudaError_t launch_fit(int C, const FitArgs& a, bool vreg, int threads, int grid, size_t smem, cudaStream_t s);
+template <int CT> const void* generic_fit_kernel(bool vreg);   // run-time strides
+template <int HSC> const void* fast_fit_kernel(bool vreg);     // compile-time strides
+
+// Kernel for a launch of fits with C classes, padded width Hs, padded feature count dp;
+// vreg: second moments of W1 in registers.  Null when C is out of range.
+const void* fit_kernel_for(int C, int Hs, int dp, bool vreg);
 
 }  // namespace bbo
