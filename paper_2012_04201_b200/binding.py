@@ -32,7 +32,7 @@ EXPORTS = [
     "bbo_mlp_cv_fold_scores", "bbo_mlp_cv_loss_trace", "bbo_mlp_cv_debug_theta",
     "bbo_mlp_cv_debug_indices", "bbo_mlp_cv_debug_rng", "bbo_mlp_cv_debug_exp",
     "bbo_mlp_cv_query_caps", "bbo_mlp_cv_last_timing", "bbo_mlp_cv_strerror",
-    "bbo_mlp_cv_last_cuda_error", "bbo_mlp_cv_eval_static",
+    "bbo_mlp_cv_last_cuda_error", "bbo_mlp_cv_eval_static", "bbo_mlp_cv_debug_fast_math",
 ]
 
 
@@ -75,6 +75,7 @@ def load():
     L.bbo_mlp_cv_debug_indices.argtypes = [vp, i64, i32, u64, i32, i32, i32, vp, vp]
     L.bbo_mlp_cv_debug_rng.argtypes = [vp, u64, vp, i64, vp]
     L.bbo_mlp_cv_debug_exp.argtypes = [vp, vp, i64, vp]
+    L.bbo_mlp_cv_debug_fast_math.argtypes = [vp, i32, u64, u64, u64, vp]
     L.bbo_mlp_cv_query_caps.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     L.bbo_mlp_cv_last_timing.argtypes = [vp, vp, vp, vp]
     L.bbo_mlp_cv_strerror.argtypes = [ctypes.c_int]
@@ -221,6 +222,12 @@ class MlpCv:
         x = np.ascontiguousarray(x, np.float32)
         out = np.empty_like(x)
         self._check(load().bbo_mlp_cv_debug_exp(self._h, _np_ptr(x), x.size, _np_ptr(out)))
+        return out
+
+    def debug_fast_math(self, mode, seed=0, first=0, count=1):
+        """(disagreements, fast-path cases, operand bits...) of the in-kernel sqrt/div check."""
+        out = np.zeros(4, np.uint64)
+        self._check(load().bbo_mlp_cv_debug_fast_math(self._h, mode, seed, first, count, _np_ptr(out)))
         return out
 
     def query_caps(self, d, n_classes):

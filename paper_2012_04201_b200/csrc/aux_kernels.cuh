@@ -65,6 +65,38 @@ __global__ void debug_rng_kernel(uint64_t seed, const uint32_t* ctr, int64_t cou
   }
 }
 
+// Debug: counts inputs in the safe range for which the branch-free square root / division
+// differ from the IEEE intrinsics.  mode 0: sqrt over the bit patterns first .. first+count-1;
+// mode 1: m / (sqrt(v) + eps) over `count` operand triples drawn from Philox words with
+// exponents spread over the whole float range.  out[0] = mismatches, out[1] = cases the fast
+// path declared safe, out[2..3] = operands of one mismatch.
+__global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, uint64_t count, unsigned long long* out) {
+  unsigned long long bad = 0, safe_n = 0;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < count; i += (uint64_t)gridDim.x * blockDim.x) {
+    if (mode == 0) {
+      const float x = __uint_as_float((uint32_t)(first + i));
+      const uint32_t xb = __float_as_uint(x);
+      if (!(((xb - kVLo) < kVSpan) || xb == 0u)) continue;
+      ++safe_n;
+      const float a = sqrt_fast_rn(x), b = __fsqrt_rn(x);
+      if (__float_as_uint(a) != __float_as_uint(b)) { ++bad; out[2] = __float_as_uint(x); }
+    } else {
+      const uint4 r = philox4x32_10(seed, 7u, (uint32_t)(i >> 32), 0u, 0u, (uint32_t)i);
+      const float m = __uint_as_float(r.x);
+      const float vv = __uint_as_float(r.y & 0x7FFFFFFFu);
+      const float eps = __uint_as_float((r.z & 0x007FFFFFu) | ((20u + (r.w % 170u)) << 23));  // 2^-107 .. 2^62
+      uint32_t safe = adam_eps_safe(eps);
+      const float q = adam_ratio_fast(m, vv, eps, safe);
+      if (safe == 0u) continue;
+      ++safe_n;
+      const float ref = adam_ratio_ieee(m, vv, eps);
+      if (__float_as_uint(q) != __float_as_uint(ref)) { ++bad; out[2] = __float_as_uint(m); out[3] = __float_as_uint(vv); }
+    }
+  }
+  if (bad) atomicAdd(&out[0], bad);
+  if (safe_n) atomicAdd(&out[1], safe_n);
+}
+
 __global__ void debug_exp_kernel(const float* x, int64_t count, float* out) {
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
     out[i] = spec_expf(x[i]);

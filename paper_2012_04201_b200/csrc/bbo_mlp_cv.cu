@@ -545,6 +545,20 @@ int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* ou
   return BBO_OK;
 }
 
+int bbo_mlp_cv_debug_fast_math(bbo_mlp_cv* h, int32_t mode, uint64_t seed, uint64_t first, uint64_t count,
+                               uint64_t* host_out4) {
+  if (!h || !host_out4 || count < 1 || (mode != 0 && mode != 1)) return BBO_ERR_INVALID_ARG;
+  DeviceGuard g(h->device);
+  cudaStream_t s = h->stream;
+  BBO_CUDA(h, h->dbg_u.reserve(8));
+  BBO_CUDA(h, cudaMemsetAsync(h->dbg_u.p, 0, 32, s));
+  bbo::debug_fast_math_kernel<<<h->sm_count * 8, 256, 0, s>>>(mode, seed, first, count, reinterpret_cast<unsigned long long*>(h->dbg_u.p));
+  BBO_CUDA(h, cudaGetLastError());
+  BBO_CUDA(h, cudaMemcpyAsync(host_out4, h->dbg_u.p, 32, cudaMemcpyDeviceToHost, s));
+  BBO_CUDA(h, cudaStreamSynchronize(s));
+  return BBO_OK;
+}
+
 int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* max_n, int32_t* max_d,
                           int32_t* max_hidden, int32_t* max_classes) {
   if (!h || d < 1 || n_classes < 1 || n_classes > kMaxClasses) return BBO_ERR_INVALID_ARG;

@@ -153,7 +153,29 @@ __device__ __forceinline__ void adam_one(float& th, float& m, float& vv, float g
                                          float omb1, float omb2, float step, float eps) {
   m = __fmaf_rn(beta1, m, __fmul_rn(omb1, g));
   vv = __fmaf_rn(beta2, vv, __fmul_rn(__fmul_rn(omb2, g), g));
-  th = __fsub_rn(th, __fmul_rn(step, __fdiv_rn(m, __fadd_rn(__fsqrt_rn(vv), eps))));
+  th = __fsub_rn(th, __fmul_rn(step, adam_ratio_ieee(m, vv, eps)));
+}
+
+// Adam on N parameters held in registers.  The N updates are independent straight-line code
+// (branch-free square root and division), with one rarely taken fallback for the whole group.
+template <int N>
+__device__ __forceinline__ void adam_group(float (&th)[N], float (&m)[N], float (&vv)[N], const float (&g)[N],
+                                           float beta1, float beta2, float omb1, float omb2, float step, float eps,
+                                           uint32_t eps_safe) {
+  float q[N];
+  uint32_t safe = eps_safe;
+#pragma unroll
+  for (int e = 0; e < N; ++e) {
+    m[e] = __fmaf_rn(beta1, m[e], __fmul_rn(omb1, g[e]));
+    vv[e] = __fmaf_rn(beta2, vv[e], __fmul_rn(__fmul_rn(omb2, g[e]), g[e]));
+    q[e] = adam_ratio_fast(m[e], vv[e], eps, safe);
+  }
+  if (safe == 0u) {
+#pragma unroll
+    for (int e = 0; e < N; ++e) q[e] = adam_ratio_ieee(m[e], vv[e], eps);
+  }
+#pragma unroll
+  for (int e = 0; e < N; ++e) th[e] = __fsub_rn(th[e], __fmul_rn(step, q[e]));
 }
 
 struct BlockShared {  // block-wide scalars
@@ -270,6 +292,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 
   const float beta1 = c.beta1, beta2 = c.beta2, eps = c.eps;
   const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
+  const uint32_t eps_safe = adam_eps_safe(eps);
   double p1 = 1.0, p2 = 1.0;  // running beta^t (thread 0 only)
   int step_no = 0;
   float v1[8][8];             // second moments of this thread's W1 tile (VR only)
@@ -415,36 +438,52 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         for (int i = 0; i < 8; ++i) {
           const int k = k0 + i;
           if (k < d) {
+            const int offA = L.oW1 + k * Hs + jA, offB = L.oW1 + k * Hs + jB;
+            const float4 wA = *reinterpret_cast<float4*>(v.W + offA), wB = *reinterpret_cast<float4*>(v.W + offB);
+            const float4 mA = *reinterpret_cast<float4*>(v.M + offA), mB = *reinterpret_cast<float4*>(v.M + offB);
+            float w8[8] = {wA.x, wA.y, wA.z, wA.w, wB.x, wB.y, wB.z, wB.w};
+            float m8[8] = {mA.x, mA.y, mA.z, mA.w, mB.x, mB.y, mB.z, mB.w};
+            float v8[8], g8[8];
+            if (VR) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const int off = L.oW1 + k * Hs + (half ? jB : jA);
-              float4 w = *reinterpret_cast<float4*>(v.W + off);
-              float4 m = *reinterpret_cast<float4*>(v.M + off);
-              float4 vv;
-              if (VR) vv = make_float4(v1[i][4 * half], v1[i][4 * half + 1], v1[i][4 * half + 2], v1[i][4 * half + 3]);
-              else vv = *reinterpret_cast<float4*>(v.V + off);
-              adam_one(w.x, m.x, vv.x, __fmaf_rn(aB, w.x, g1[i][4 * half]), beta1, beta2, omb1, omb2, step, eps);
-              adam_one(w.y, m.y, vv.y, __fmaf_rn(aB, w.y, g1[i][4 * half + 1]), beta1, beta2, omb1, omb2, step, eps);
-              adam_one(w.z, m.z, vv.z, __fmaf_rn(aB, w.z, g1[i][4 * half + 2]), beta1, beta2, omb1, omb2, step, eps);
-              adam_one(w.w, m.w, vv.w, __fmaf_rn(aB, w.w, g1[i][4 * half + 3]), beta1, beta2, omb1, omb2, step, eps);
-              *reinterpret_cast<float4*>(v.W + off) = w;
-              *reinterpret_cast<float4*>(v.M + off) = m;
-              if (VR) { v1[i][4 * half] = vv.x; v1[i][4 * half + 1] = vv.y; v1[i][4 * half + 2] = vv.z; v1[i][4 * half + 3] = vv.w; }
-              else *reinterpret_cast<float4*>(v.V + off) = vv;
+              for (int j = 0; j < 8; ++j) v8[j] = v1[i][j];
+            } else {
+              const float4 vA = *reinterpret_cast<float4*>(v.V + offA), vB = *reinterpret_cast<float4*>(v.V + offB);
+              v8[0] = vA.x; v8[1] = vA.y; v8[2] = vA.z; v8[3] = vA.w; v8[4] = vB.x; v8[5] = vB.y; v8[6] = vB.z; v8[7] = vB.w;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) g8[j] = __fmaf_rn(aB, w8[j], g1[i][j]);
+            adam_group<8>(w8, m8, v8, g8, beta1, beta2, omb1, omb2, step, eps, eps_safe);
+            *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
+            *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
+            *reinterpret_cast<float4*>(v.M + offA) = make_float4(m8[0], m8[1], m8[2], m8[3]);
+            *reinterpret_cast<float4*>(v.M + offB) = make_float4(m8[4], m8[5], m8[6], m8[7]);
+            if (VR) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v1[i][j] = v8[j];
+            } else {
+              *reinterpret_cast<float4*>(v.V + offA) = make_float4(v8[0], v8[1], v8[2], v8[3]);
+              *reinterpret_cast<float4*>(v.V + offB) = make_float4(v8[4], v8[5], v8[6], v8[7]);
             }
           }
         }
       }
       if (unit_role) {
+        float wu[CT + 1], mu[CT + 1], vu[CT + 1], gu[CT + 1];
 #pragma unroll
         for (int o = 0; o < CT; ++o) {
           const int off = L.oW2 + tid * CS + o;
-          float w = w2[o];
-          adam_one(w, v.M[off], v.V[off], __fmaf_rn(aB, w, g2[o]), beta1, beta2, omb1, omb2, step, eps);
-          v.W[off] = w;
+          wu[o] = w2[o]; mu[o] = v.M[off]; vu[o] = v.V[off];
+          gu[o] = __fmaf_rn(aB, w2[o], g2[o]);
         }
-        const int off = L.ob1 + tid;
-        adam_one(v.W[off], v.M[off], v.V[off], gb1, beta1, beta2, omb1, omb2, step, eps);
+        wu[CT] = v.W[L.ob1 + tid]; mu[CT] = v.M[L.ob1 + tid]; vu[CT] = v.V[L.ob1 + tid]; gu[CT] = gb1;
+        adam_group<CT + 1>(wu, mu, vu, gu, beta1, beta2, omb1, omb2, step, eps, eps_safe);
+#pragma unroll
+        for (int o = 0; o < CT; ++o) {
+          const int off = L.oW2 + tid * CS + o;
+          v.W[off] = wu[o]; v.M[off] = mu[o]; v.V[off] = vu[o];
+        }
+        v.W[L.ob1 + tid] = wu[CT]; v.M[L.ob1 + tid] = mu[CT]; v.V[L.ob1 + tid] = vu[CT];
       }
       if (o_role) {
         const int off = L.ob2 + tid;

@@ -88,6 +88,22 @@ def test_exponential_bit_exact(binding):
     assert np.isnan(got[-4]) and got[-3] == 0.0 and np.isinf(got[-2]) and got[-1] == 1.0
 
 
+def test_branch_free_sqrt_and_division_equal_ieee(binding):
+    h = binding.MlpCv()
+    # every non-negative float bit pattern (zero, denormals, normals, inf, NaN): the fast path
+    # must agree with the IEEE square root wherever it claims to be valid
+    out = h.debug_fast_math(0, first=0, count=2**31)
+    assert out[0] == 0 and out[1] > 1.6e9, out
+    # 2^32 operand triples with exponents across the whole range
+    total_safe = 0
+    for seed in (1, 2):
+        out = h.debug_fast_math(1, seed=seed, count=2**31)
+        assert out[0] == 0, out
+        total_safe += int(out[1])
+    assert total_safe > 5e7
+    h.close()
+
+
 @pytest.mark.parametrize("n,K", [(150, 5), (569, 5), (1797, 5), (442, 5), (37, 3), (12, 12), (4100, 7)])
 def test_fold_split_and_minibatch_order_bit_exact(binding, n, K):
     h = binding.MlpCv()
