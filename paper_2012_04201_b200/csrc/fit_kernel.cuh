@@ -365,20 +365,43 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         // ---- hidden unit tid: gW2[tid][:], delta1[:, tid] in place over A1, gb1[tid]; b ascending ----
         if (unit_role) {
           float* ap = v.A1 + tid;
-#pragma unroll 2
-          for (int b = 0; b < nb; ++b) {
-            const float a1 = ap[b * Hs];
-            float dl[(CT + 3) / 4 * 4];
+          constexpr int C4 = (CT + 3) / 4;
+          int b = 0;
+          for (; b + 4 <= nb; b += 4) {  // four rows at a time: loads first, then four independent delta1 chains
+            float a1r[4], dl[4][C4 * 4], acc[4];
 #pragma unroll
-            for (int o4 = 0; o4 < (CT + 3) / 4; ++o4) {
-              const float4 t = *reinterpret_cast<const float4*>(v.D2 + b * CS + 4 * o4);
-              dl[4 * o4] = t.x; dl[4 * o4 + 1] = t.y; dl[4 * o4 + 2] = t.z; dl[4 * o4 + 3] = t.w;
+            for (int r = 0; r < 4; ++r) {
+              a1r[r] = ap[(b + r) * Hs];
+#pragma unroll
+              for (int o4 = 0; o4 < C4; ++o4) {
+                const float4 t = *reinterpret_cast<const float4*>(v.D2 + (b + r) * CS + 4 * o4);
+                dl[r][4 * o4] = t.x; dl[r][4 * o4 + 1] = t.y; dl[r][4 * o4 + 2] = t.z; dl[r][4 * o4 + 3] = t.w;
+              }
+              acc[r] = 0.f;
             }
+#pragma unroll
+            for (int o = 0; o < CT; ++o) {
+#pragma unroll
+              for (int r = 0; r < 4; ++r) {
+                g2[o] = __fmaf_rn(a1r[r], dl[r][o], g2[o]);
+                acc[r] = __fmaf_rn(dl[r][o], w2[o], acc[r]);
+              }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              const float d1 = a1r[r] > 0.f ? acc[r] : 0.f;
+              ap[(b + r) * Hs] = d1;
+              gb1 = __fadd_rn(gb1, d1);
+            }
+          }
+          for (; b < nb; ++b) {
+            const float a1 = ap[b * Hs];
             float acc = 0.f;
 #pragma unroll
             for (int o = 0; o < CT; ++o) {
-              g2[o] = __fmaf_rn(a1, dl[o], g2[o]);
-              acc = __fmaf_rn(dl[o], w2[o], acc);
+              const float dv = v.D2[b * CS + o];
+              g2[o] = __fmaf_rn(a1, dv, g2[o]);
+              acc = __fmaf_rn(dv, w2[o], acc);
             }
             const float d1 = a1 > 0.f ? acc : 0.f;
             ap[b * Hs] = d1;
