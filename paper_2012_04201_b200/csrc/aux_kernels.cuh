@@ -47,9 +47,10 @@ __global__ void debug_order_kernel(int n, int K, uint64_t seed, const int32_t* p
   int vb, vs;
   fold_segment(n, K, fold, &vb, &vs);
   const int n_tr = n - vs;
+  __shared__ uint32_t red[32];
   uint16_t* order = reinterpret_cast<uint16_t*>(smem);
-  uint64_t* keys = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(smem) + round_up(2 * n_tr, 16));
-  build_epoch_order(keys, order, pi, n_tr, vb, vs, seed, config, fold, epoch, threadIdx.x, blockDim.x);
+  void* scratch = reinterpret_cast<char*>(smem) + round_up(2 * n_tr, 16);
+  build_epoch_order(scratch, red, order, pi, n_tr, vb, vs, seed, config, fold, epoch, threadIdx.x, blockDim.x);
   for (int i = threadIdx.x; i < n_tr; i += blockDim.x) order_out[i] = order[i];
   for (int f = 0; f < K; ++f) {
     int b, s;

@@ -507,7 +507,7 @@ int bbo_mlp_cv_debug_indices(bbo_mlp_cv* h, int64_t n64, int32_t K, uint64_t see
   int vb, vs;
   bbo::fold_segment(n, K, fold, &vb, &vs);
   const int n_tr = n - vs;
-  const size_t bytes = (size_t)bbo::round_up(2 * n_tr, 16) + 8u * (size_t)bbo::next_pow2(n_tr);
+  const size_t bytes = (size_t)bbo::round_up(2 * n_tr, 16) + bbo::sort_scratch_bytes(n_tr);
   BBO_CUDA(h, cudaFuncSetAttribute(bbo::debug_order_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
   bbo::debug_order_kernel<<<1, 256, bytes, s>>>(n, K, seed, h->pi.p, config, fold, epoch, h->dbg_i.p, h->dbg_i.p + n);
   BBO_CUDA(h, cudaGetLastError());

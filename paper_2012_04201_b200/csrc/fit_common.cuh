@@ -54,6 +54,11 @@ __host__ __device__ inline int next_pow2(int x) {
   return p;
 }
 
+constexpr int kSortBuckets = 2048;  // power of two
+
+// Scratch of the in-kernel permutation: one 64-bit key per element plus the bucket counters.
+__host__ __device__ inline size_t sort_scratch_bytes(int n) { return 8u * (size_t)round_up(n, 2) + 4u * kSortBuckets; }
+
 // Dynamic shared memory of one fit.  vreg: second moments of W1 live in registers.
 __host__ __device__ inline size_t fit_smem_bytes(int d, int dp, int Hs, int CS, int TB, int order_bytes,
                                                  int loss_cap, int n_sort, bool vreg) {
@@ -61,7 +66,7 @@ __host__ __device__ inline size_t fit_smem_bytes(int d, int dp, int Hs, int CS, 
   size_t bytes = 4u * (size_t)(2 * L.PS + (vreg ? L.PT : L.PS));
   bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + 8u * TB + 4u * (size_t)TB * CS;
   const size_t xa = 8u * (size_t)TB * dp + 4u * (size_t)TB * Hs;
-  const size_t keys = 8u * (size_t)next_pow2(n_sort);
+  const size_t keys = sort_scratch_bytes(n_sort);
   return bytes + (xa > keys ? xa : keys);
 }
 
@@ -115,12 +120,78 @@ __device__ inline void sorted_keys(uint64_t* keys, int N, uint64_t seed, uint32_
   bitonic_sort(keys, np2, tid, nt);
 }
 
+// Permutation of 0..N-1 by ascending (random word << 32 | index), for the fit kernel: the
+// words are bucketed by their top bits (counting sort with shared-memory atomics), and each
+// bucket, which holds about N / kSortBuckets keys, is ordered by insertion.  The result is the
+// unique ascending order of the keys, whatever order the atomics ran in.  scratch:
+// sort_scratch_bytes(N) bytes, 8-byte aligned.  The sorted keys are left in keys[0..N); the
+// block is synchronised on return.  red: 32 words of shared memory.
+__device__ inline uint64_t* bucket_sorted_keys(void* scratch, uint32_t* red, int N, uint64_t seed, uint32_t stream,
+                                               uint32_t a, uint32_t b, uint32_t c, int tid, int nt) {
+  uint64_t* keys = reinterpret_cast<uint64_t*>(scratch);
+  uint32_t* cnt = reinterpret_cast<uint32_t*>(keys + round_up(N, 2));
+  constexpr int shift = 32 - 11;
+  static_assert(kSortBuckets == (1 << 11), "bucket index uses the top 11 bits");
+  const int n_blk = (N + 3) >> 2;
+  for (int i = tid; i < kSortBuckets; i += nt) cnt[i] = 0u;
+  __syncthreads();
+  for (int blk = tid; blk < n_blk; blk += nt) {  // count
+    const uint4 r = philox4x32_10(seed, stream, a, b, c, (uint32_t)blk);
+#pragma unroll
+    for (int w = 0; w < 4; ++w)
+      if (4 * blk + w < N) atomicAdd(&cnt[word_of(r, w) >> shift], 1u);
+  }
+  __syncthreads();
+  {  // exclusive scan of the counters, in place
+    const int chunk = (kSortBuckets + nt - 1) / nt;
+    const int lo = tid * chunk, hi = (lo + chunk) < kSortBuckets ? (lo + chunk) : kSortBuckets;
+    uint32_t sum = 0u;
+    for (int i = lo; i < hi; ++i) sum += cnt[i];
+    uint32_t incl = sum;
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += t;
+    }
+    if (lane == 31) red[warp] = incl;
+    __syncthreads();
+    uint32_t base = incl - sum;
+    for (int w = 0; w < warp; ++w) base += red[w];
+    for (int i = lo; i < hi; ++i) { const uint32_t t = cnt[i]; cnt[i] = base; base += t; }
+  }
+  __syncthreads();
+  for (int blk = tid; blk < n_blk; blk += nt) {  // scatter; afterwards cnt[k] = end of bucket k
+    const uint4 r = philox4x32_10(seed, stream, a, b, c, (uint32_t)blk);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const int i = 4 * blk + w;
+      if (i < N) {
+        const uint32_t word = word_of(r, w);
+        const uint32_t slot = atomicAdd(&cnt[word >> shift], 1u);
+        keys[slot] = ((uint64_t)word << 32) | (uint32_t)i;
+      }
+    }
+  }
+  __syncthreads();
+  for (int k = tid; k < kSortBuckets; k += nt) {  // order each bucket
+    const int lo = k == 0 ? 0 : (int)cnt[k - 1], hi = (int)cnt[k];
+    for (int i = lo + 1; i < hi; ++i) {
+      const uint64_t x = keys[i];
+      int j = i - 1;
+      while (j >= lo && keys[j] > x) { keys[j + 1] = keys[j]; --j; }
+      keys[j + 1] = x;
+    }
+  }
+  __syncthreads();
+  return keys;
+}
+
 // Dataset row visited i-th in epoch `epoch`: the epoch permutation applied to the training
 // list (fold permutation with the held-out segment removed, order kept).
-__device__ inline void build_epoch_order(uint64_t* keys, uint16_t* order, const int32_t* pi, int n_tr,
+__device__ inline void build_epoch_order(void* scratch, uint32_t* red, uint16_t* order, const int32_t* pi, int n_tr,
                                          int vb, int vs, uint64_t seed, uint32_t config, uint32_t fold,
                                          uint32_t epoch, int tid, int nt) {
-  sorted_keys(keys, n_tr, seed, kStreamPerm, config, fold, epoch, tid, nt);
+  const uint64_t* keys = bucket_sorted_keys(scratch, red, n_tr, seed, kStreamPerm, config, fold, epoch, tid, nt);
   for (int i = tid; i < n_tr; i += nt) {
     const int s = (int)(uint32_t)keys[i];
     order[i] = (uint16_t)pi[s < vb ? s : s + vs];

@@ -302,7 +302,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     for (int j = 0; j < 8; ++j) v1[i][j] = 0.f;
 
   for (int e = 0; e < c.epochs; ++e) {
-    build_epoch_order(v.keys, v.order, a.pi, n_tr, vb, vs, a.seed, config, fold, e, tid, nt);
+    build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, vs, a.seed, config, fold, e, tid, nt);
     int buf = 0;
     {  // first sub-tile of the epoch
       const int Bs0 = n_tr < B ? n_tr : B, nb0 = Bs0 < TB ? Bs0 : TB;
