@@ -67,7 +67,7 @@ __global__ void debug_rng_kernel(uint64_t seed, const uint32_t* ctr, int64_t cou
 }
 
 // Debug: counts inputs in the safe range for which the branch-free square root / division
-// differ from the IEEE intrinsics.  mode 0: sqrt over the bit patterns first .. first+count-1;
+// differ from the IEEE intrinsics.  mode 0: sqrt(v) and sqrt(v) + eps over the bit patterns first .. first+count-1 (denormals included);
 // mode 1: m / (sqrt(v) + eps) over `count` operand triples drawn from Philox words with
 // exponents spread over the whole float range.  out[0] = mismatches, out[1] = cases the fast
 // path declared safe, out[2..3] = operands of one mismatch.
@@ -76,11 +76,12 @@ __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, 
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < count; i += (uint64_t)gridDim.x * blockDim.x) {
     if (mode == 0) {
       const float x = __uint_as_float((uint32_t)(first + i));
-      const uint32_t xb = __float_as_uint(x);
-      if (!(((xb - kVLo) < kVSpan) || xb == 0u)) continue;
+      if (__float_as_uint(x) >= kVHi) continue;
       ++safe_n;
-      const float a = sqrt_fast_rn(x), b = __fsqrt_rn(x);
-      if (__float_as_uint(a) != __float_as_uint(b)) { ++bad; out[2] = __float_as_uint(x); }
+      const float eps = 0x1p-30f;
+      const float a = adam_denominator_fast(x, eps), b = __fadd_rn(__fsqrt_rn(x), eps);
+      const float a2 = __fmul_rn(sqrt_fast_rn(fmaxf(__fmul_rn(x, 0x1p+96f), 0x1p-60f)), 0x1p-48f), b2 = __fsqrt_rn(x);
+      if (__float_as_uint(a) != __float_as_uint(b) || (x != 0.f && __float_as_uint(a2) != __float_as_uint(b2))) { ++bad; out[2] = __float_as_uint(x); }
     } else {
       const uint4 r = philox4x32_10(seed, 7u, (uint32_t)(i >> 32), 0u, 0u, (uint32_t)i);
       const float m = __uint_as_float(r.x);

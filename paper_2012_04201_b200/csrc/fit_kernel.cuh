@@ -156,26 +156,37 @@ __device__ __forceinline__ void adam_one(float& th, float& m, float& vv, float g
   th = __fsub_rn(th, __fmul_rn(step, adam_ratio_ieee(m, vv, eps)));
 }
 
-// Adam on N parameters held in registers.  The N updates are independent straight-line code
-// (branch-free square root and division), with one rarely taken fallback for the whole group.
+// Adam on N parameters held in registers, first pass: moments updated in place, parameters
+// updated with the branch-free ratio.  Returns 1 when every ratio was computed inside the range
+// in which it equals the IEEE result; otherwise the caller discards th[] and redoes the
+// parameter update with adam_params_ieee from the updated moments.
 template <int N>
-__device__ __forceinline__ void adam_group(float (&th)[N], float (&m)[N], float (&vv)[N], const float (&g)[N],
-                                           float beta1, float beta2, float omb1, float omb2, float step, float eps,
-                                           uint32_t eps_safe) {
-  float q[N];
+__device__ __forceinline__ uint32_t adam_group_fast(float (&th)[N], float (&m)[N], float (&vv)[N], const float (&g)[N],
+                                                    float beta1, float beta2, float omb1, float omb2, float step,
+                                                    float eps, uint32_t eps_safe) {
   uint32_t safe = eps_safe;
 #pragma unroll
   for (int e = 0; e < N; ++e) {
     m[e] = __fmaf_rn(beta1, m[e], __fmul_rn(omb1, g[e]));
     vv[e] = __fmaf_rn(beta2, vv[e], __fmul_rn(__fmul_rn(omb2, g[e]), g[e]));
-    q[e] = adam_ratio_fast(m[e], vv[e], eps, safe);
+    th[e] = __fsub_rn(th[e], __fmul_rn(step, adam_ratio_fast(m[e], vv[e], eps, safe)));
   }
-  if (safe == 0u) {
+  return safe;
+}
+
+// Second pass for a group the first pass could not certify: IEEE square root and division.
+// A NaN moment gives NaN either way, and skipping the library call there keeps fits whose
+// parameters have become NaN at full speed.
+template <int N>
+__device__ __forceinline__ void adam_params_ieee(float (&th)[N], const float (&m)[N], const float (&vv)[N], float step,
+                                                 float eps) {
 #pragma unroll
-    for (int e = 0; e < N; ++e) q[e] = adam_ratio_ieee(m[e], vv[e], eps);
+  for (int e = 0; e < N; ++e) {
+    float q;
+    if (m[e] != m[e] || vv[e] != vv[e]) q = __fadd_rn(m[e], vv[e]);
+    else q = adam_ratio_ieee(m[e], vv[e], eps);
+    th[e] = __fsub_rn(th[e], __fmul_rn(step, q));
   }
-#pragma unroll
-  for (int e = 0; e < N; ++e) th[e] = __fsub_rn(th[e], __fmul_rn(step, q[e]));
 }
 
 struct BlockShared {  // block-wide scalars
@@ -199,7 +210,7 @@ __device__ __forceinline__ float row_delta(const FitView& v, int task, float z, 
     float sum = 0.f;
 #pragma unroll
     for (int o = 0; o < CT; ++o) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, ex, obase + o));
-    const float pr = __fdiv_rn(ex, sum);
+    const float pr = sum != sum ? sum : __fdiv_rn(ex, sum);  // NaN row: skip the library's special-case path
     if (want_loss) {
       const float zl = __shfl_sync(0xffffffffu, z, obase + (active ? label : 0));
       if (active && ocol == 0) v.lossb[loss_idx] = __fsub_rn(logf(sum), __fsub_rn(zl, mx));
@@ -457,6 +468,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       // ---- L2 term and Adam, by the owner of each gradient ----
       const float step = sh.step[step_no & 1];
       if (has_tile) {
+        uint32_t redo = 0u;  // rows of the tile whose fast update could not be certified
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int k = k0 + i;
@@ -476,9 +488,13 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
             }
 #pragma unroll
             for (int j = 0; j < 8; ++j) g8[j] = __fmaf_rn(aB, w8[j], g1[i][j]);
-            adam_group<8>(w8, m8, v8, g8, beta1, beta2, omb1, omb2, step, eps, eps_safe);
-            *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
-            *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
+            const uint32_t safe = adam_group_fast<8>(w8, m8, v8, g8, beta1, beta2, omb1, omb2, step, eps, eps_safe);
+            if (safe) {
+              *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
+              *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
+            } else {
+              redo |= 1u << i;
+            }
             *reinterpret_cast<float4*>(v.M + offA) = make_float4(m8[0], m8[1], m8[2], m8[3]);
             *reinterpret_cast<float4*>(v.M + offB) = make_float4(m8[4], m8[5], m8[6], m8[7]);
             if (VR) {
@@ -490,9 +506,32 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
             }
           }
         }
+        if (redo) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (redo & (1u << i)) {
+              const int offA = L.oW1 + (k0 + i) * Hs + jA, offB = L.oW1 + (k0 + i) * Hs + jB;
+              const float4 wA = *reinterpret_cast<float4*>(v.W + offA), wB = *reinterpret_cast<float4*>(v.W + offB);
+              const float4 mA = *reinterpret_cast<float4*>(v.M + offA), mB = *reinterpret_cast<float4*>(v.M + offB);
+              float w8[8] = {wA.x, wA.y, wA.z, wA.w, wB.x, wB.y, wB.z, wB.w};
+              const float m8[8] = {mA.x, mA.y, mA.z, mA.w, mB.x, mB.y, mB.z, mB.w};
+              float v8[8];
+              if (VR) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v8[j] = v1[i][j];
+              } else {
+                const float4 vA = *reinterpret_cast<float4*>(v.V + offA), vB = *reinterpret_cast<float4*>(v.V + offB);
+                v8[0] = vA.x; v8[1] = vA.y; v8[2] = vA.z; v8[3] = vA.w; v8[4] = vB.x; v8[5] = vB.y; v8[6] = vB.z; v8[7] = vB.w;
+              }
+              adam_params_ieee<8>(w8, m8, v8, step, eps);
+              *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
+              *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
+            }
+          }
+        }
       }
       if (unit_role) {
-        float wu[CT + 1], mu[CT + 1], vu[CT + 1], gu[CT + 1];
+        float wu[CT + 1], mu[CT + 1], vu[CT + 1], gu[CT + 1], wold[CT + 1];
 #pragma unroll
         for (int o = 0; o < CT; ++o) {
           const int off = L.oW2 + tid * CS + o;
@@ -500,7 +539,13 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           gu[o] = __fmaf_rn(aB, w2[o], g2[o]);
         }
         wu[CT] = v.W[L.ob1 + tid]; mu[CT] = v.M[L.ob1 + tid]; vu[CT] = v.V[L.ob1 + tid]; gu[CT] = gb1;
-        adam_group<CT + 1>(wu, mu, vu, gu, beta1, beta2, omb1, omb2, step, eps, eps_safe);
+#pragma unroll
+        for (int o = 0; o <= CT; ++o) wold[o] = wu[o];
+        if (!adam_group_fast<CT + 1>(wu, mu, vu, gu, beta1, beta2, omb1, omb2, step, eps, eps_safe)) {
+#pragma unroll
+          for (int o = 0; o <= CT; ++o) wu[o] = wold[o];
+          adam_params_ieee<CT + 1>(wu, mu, vu, step, eps);
+        }
 #pragma unroll
         for (int o = 0; o < CT; ++o) {
           const int off = L.oW2 + tid * CS + o;
