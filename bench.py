@@ -200,7 +200,7 @@ def workload_config(args, wl, work):
     return {"workload": "digits_sweep", "n": int(wl["X"].shape[0]), "d": int(wl["X"].shape[1]), "classes": 10,
             "n_folds": 5, "epochs": int(args.epochs), "fits_per_step": int(work["n_fits"]),
             "hidden": args.hidden or "U{50..200}", "batch_size": args.batch or "U{10..250}",
-            "l2_between_steps": "flushed (256 MiB write)", "variant": "fp32-cuda-core"}
+            "l2_between_steps": "flushed (256 MiB write)", "variant": "fp32-cuda-core, one CTA per fit, one launch per hidden-width group"}
 
 
 def main():
@@ -311,6 +311,13 @@ def main():
     }
     if clocks.get("sm_mhz"):
         roofline["frac_at_sampled_clock"] = achieved / (fp32_peak * clocks["sm_mhz"] / sm_max)
+    try:  # FMA rate this device sustains from registers, measured now
+        ffma = h.debug_ffma_peak()
+        roofline["peak_measured_ffma"] = ffma
+        roofline["frac_of_measured_ffma"] = achieved / ffma
+    except Exception as exc:  # pragma: no cover
+        roofline["peak_measured_ffma"] = None
+        roofline["peak_measured_ffma_error"] = str(exc)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -66,7 +66,11 @@ typedef struct {
   int32_t keep_theta;  /* 1: keep the final parameters of the LAST fit of the list, i.e.
                           (configuration n_configs-1, fold n_folds-1), for
                           bbo_mlp_cv_debug_theta                                            */
-  int32_t reserved[3];
+  int32_t config_index_base; /* added to each configuration's position in the list when keying
+                          its random streams: a caller that splits one params_list over several
+                          handles (e.g. one per GPU) passes the position of its first entry and
+                          gets the scores the unsplit call would give                          */
+  int32_t reserved[2];
 } bbo_mlp_cv_options;
 
 /* Creates a handle bound to one device and one stream.  `opt` may be NULL (defaults).
@@ -131,6 +135,12 @@ int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* ou
  * operand bits of one disagreement.                                                       */
 int bbo_mlp_cv_debug_fast_math(bbo_mlp_cv* h, int32_t mode, uint64_t seed, uint64_t first,
                                uint64_t count, uint64_t* host_out4);
+
+/* Measures the FP32 fused-multiply-add rate this device sustains from registers (no memory
+ * traffic): every SM runs `threads_per_sm` threads doing `iters` rounds of 16 independent
+ * FMAs.  *tflops receives 2 * FMAs / time.  It is the roofline ceiling the fit kernel is
+ * compared with, measured at the clock the device actually holds.                          */
+int bbo_mlp_cv_debug_ffma_peak(bbo_mlp_cv* h, int32_t threads_per_sm, int32_t iters, float* tflops);
 
 /* Largest shapes one call accepts on this device: rows, features, hidden width for the
  * given (d, n_classes) pair, and classes.  Any output pointer may be NULL.               */

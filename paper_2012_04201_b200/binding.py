@@ -32,14 +32,14 @@ EXPORTS = [
     "bbo_mlp_cv_fold_scores", "bbo_mlp_cv_loss_trace", "bbo_mlp_cv_debug_theta",
     "bbo_mlp_cv_debug_indices", "bbo_mlp_cv_debug_rng", "bbo_mlp_cv_debug_exp",
     "bbo_mlp_cv_query_caps", "bbo_mlp_cv_last_timing", "bbo_mlp_cv_strerror",
-    "bbo_mlp_cv_last_cuda_error", "bbo_mlp_cv_eval_static", "bbo_mlp_cv_debug_fast_math",
+    "bbo_mlp_cv_last_cuda_error", "bbo_mlp_cv_eval_static", "bbo_mlp_cv_debug_fast_math", "bbo_mlp_cv_debug_ffma_peak",
 ]
 
 
 class Options(ctypes.Structure):
     _fields_ = [("device", ctypes.c_int32), ("stream", ctypes.c_void_p), ("n_classes", ctypes.c_int32),
                 ("trace_steps", ctypes.c_int32), ("keep_theta", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 3)]
+                ("config_index_base", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
 
 
 _lib = None
@@ -76,6 +76,7 @@ def load():
     L.bbo_mlp_cv_debug_rng.argtypes = [vp, u64, vp, i64, vp]
     L.bbo_mlp_cv_debug_exp.argtypes = [vp, vp, i64, vp]
     L.bbo_mlp_cv_debug_fast_math.argtypes = [vp, i32, u64, u64, u64, vp]
+    L.bbo_mlp_cv_debug_ffma_peak.argtypes = [vp, i32, i32, vp]
     L.bbo_mlp_cv_query_caps.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     L.bbo_mlp_cv_last_timing.argtypes = [vp, vp, vp, vp]
     L.bbo_mlp_cv_strerror.argtypes = [ctypes.c_int]
@@ -101,9 +102,9 @@ def _np_ptr(a):
 
 
 # ---- functions with the C names -------------------------------------------------------
-def bbo_mlp_cv_create(device=-1, stream=0, n_classes=0, trace_steps=0, keep_theta=0):
+def bbo_mlp_cv_create(device=-1, stream=0, n_classes=0, trace_steps=0, keep_theta=0, config_index_base=0):
     opt = Options(device=device, stream=stream or None, n_classes=n_classes, trace_steps=trace_steps,
-                  keep_theta=int(keep_theta))
+                  keep_theta=int(keep_theta), config_index_base=int(config_index_base))
     h = ctypes.c_void_p()
     rc = load().bbo_mlp_cv_create(ctypes.byref(opt), ctypes.byref(h))
     if rc != BBO_OK:
@@ -142,7 +143,7 @@ def bbo_mlp_cv_eval_static(stream_ptr, X_ptr, y_ptr, n, d, task, n_folds, n_clas
 class MlpCv:
     """One handle = one device, one stream, one call in flight."""
 
-    def __init__(self, device=None, stream=None, n_classes=0, trace_steps=0, keep_theta=False):
+    def __init__(self, device=None, stream=None, n_classes=0, trace_steps=0, keep_theta=False, config_index_base=0):
         import torch
 
         if not torch.cuda.is_available():
@@ -154,7 +155,7 @@ class MlpCv:
             torch.zeros(1, device="cuda")  # make sure the primary context exists
         self.stream = stream
         sptr = 0 if stream is None else int(stream.cuda_stream)
-        self._h = bbo_mlp_cv_create(self.device, sptr, n_classes, trace_steps, keep_theta)
+        self._h = bbo_mlp_cv_create(self.device, sptr, n_classes, trace_steps, keep_theta, config_index_base)
         self._n_configs = self._n_folds = 0
         self.trace_steps = trace_steps
 
@@ -229,6 +230,12 @@ class MlpCv:
         out = np.zeros(4, np.uint64)
         self._check(load().bbo_mlp_cv_debug_fast_math(self._h, mode, seed, first, count, _np_ptr(out)))
         return out
+
+    def debug_ffma_peak(self, threads_per_sm=1024, iters=20000):
+        """FP32 FMA rate (TFLOP/s) the device sustains from registers."""
+        out = ctypes.c_float()
+        self._check(load().bbo_mlp_cv_debug_ffma_peak(self._h, threads_per_sm, iters, ctypes.byref(out)))
+        return out.value
 
     def query_caps(self, d, n_classes):
         v = [ctypes.c_int32() for _ in range(4)]

@@ -99,6 +99,22 @@ __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, 
   if (safe_n) atomicAdd(&out[1], safe_n);
 }
 
+// Register-only FMA loop: 16 independent accumulators per thread, `iters` rounds.
+__global__ void ffma_peak_kernel(float* out, int iters) {
+  float acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc[i] = 0.001f * (float)threadIdx.x + (float)i;
+  const float x = 1.0001f, y = 0.5f;
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = __fmaf_rn(acc[i], x, y);
+  }
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) sum += acc[i];
+  out[blockIdx.x * blockDim.x + threadIdx.x] = sum;
+}
+
 __global__ void debug_exp_kernel(const float* x, int64_t count, float* out) {
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
     out[i] = spec_expf(x[i]);

@@ -196,7 +196,7 @@ struct FitBuffers {  // device scratch of one evaluation
 // (widest first; groups overlap on the side streams when there are any).
 int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk, const float* y, int n, int d,
                     int C, int K, int task, const bbo_mlp_config* configs, int n_configs, uint64_t seed,
-                    int trace_steps, int maxB, int* launches, cudaError_t* cuda_err) {
+                    int trace_steps, int maxB, int config_base, int* launches, cudaError_t* cuda_err) {
   *cuda_err = cudaSuccess;
   const int n_fits = n_configs * K;
   struct Item { int Hs; double cost; int id; };
@@ -248,7 +248,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     bbo::FitArgs a{};
     a.X = Xk; a.y = y; a.pi = buf.pi; a.configs = buf.configs; a.fits = buf.fits + g.begin;
     a.fold_scores = buf.fold_scores; a.trace = buf.trace; a.keep_theta = buf.keep_theta;
-    a.n_fits = g.count; a.n_configs = n_configs;
+    a.n_fits = g.count; a.n_configs = n_configs; a.config_base = config_base;
     a.n = n; a.d = d; a.dp = g.plan.dp; a.C = C; a.CS = g.plan.CS; a.K = K; a.task = task;
     a.Hs = g.plan.Hs; a.TB = g.plan.TB; a.trace_steps = trace_steps; a.loss_cap = g.plan.loss_cap;
     a.order_bytes = g.plan.order_bytes; a.seed = seed;
@@ -308,7 +308,8 @@ int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out) {
   }
   int dev = o.device;
   if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return BBO_ERR_CUDA;
-  if (dev >= count || o.n_classes < 0 || o.n_classes > kMaxClasses || o.trace_steps < 0) return BBO_ERR_INVALID_ARG;
+  if (dev >= count || o.n_classes < 0 || o.n_classes > kMaxClasses || o.trace_steps < 0 || o.config_index_base < 0)
+    return BBO_ERR_INVALID_ARG;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return BBO_ERR_CUDA;
   if (prop.major != 10) return BBO_ERR_UNSUPPORTED;  // the kernels are built for sm_100a only
@@ -363,7 +364,8 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   if (!h || !X || !y || !configs || !out_scores) return BBO_ERR_INVALID_ARG;
   if (n64 < 2 || d < 1 || K < 2 || K > n64 || n_configs < 1) return BBO_ERR_INVALID_ARG;
   if (task != BBO_TASK_CLASSIFICATION && task != BBO_TASK_REGRESSION) return BBO_ERR_INVALID_ARG;
-  if (n64 > kMaxRows || (int64_t)n_configs * K > (1 << 30) || n_configs >= (1 << 28)) return BBO_ERR_UNSUPPORTED;
+  if (n64 > kMaxRows || (int64_t)n_configs * K > (1 << 30) || (int64_t)n_configs + h->opt.config_index_base >= (1 << 28))
+    return BBO_ERR_UNSUPPORTED;
   int maxH, maxB;
   int rc = check_configs(configs, n_configs, &maxH, &maxB);
   if (rc != BBO_OK) return rc;
@@ -439,7 +441,7 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   BBO_CUDA(h, cudaEventRecord(h->evf0, s));
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, h->opt.trace_steps, maxB,
-                       &launches, &cuda_err);
+                       h->opt.config_index_base, &launches, &cuda_err);
   if (rc == BBO_ERR_CUDA) return cuda_fail(h, cuda_err, "launch_all_fits");
   if (rc != BBO_OK) return rc;
   BBO_CUDA(h, cudaEventRecord(h->evf1, s));
@@ -556,6 +558,24 @@ int bbo_mlp_cv_debug_fast_math(bbo_mlp_cv* h, int32_t mode, uint64_t seed, uint6
   BBO_CUDA(h, cudaGetLastError());
   BBO_CUDA(h, cudaMemcpyAsync(host_out4, h->dbg_u.p, 32, cudaMemcpyDeviceToHost, s));
   BBO_CUDA(h, cudaStreamSynchronize(s));
+  return BBO_OK;
+}
+
+int bbo_mlp_cv_debug_ffma_peak(bbo_mlp_cv* h, int32_t threads_per_sm, int32_t iters, float* tflops) {
+  if (!h || !tflops || threads_per_sm < 32 || threads_per_sm > 1024 || threads_per_sm % 32 != 0 || iters < 1)
+    return BBO_ERR_INVALID_ARG;
+  DeviceGuard g(h->device);
+  cudaStream_t s = h->stream;
+  BBO_CUDA(h, h->dbg_f.reserve((size_t)h->sm_count * threads_per_sm));
+  bbo::ffma_peak_kernel<<<h->sm_count, threads_per_sm, 0, s>>>(h->dbg_f.p, 100);  // warm-up
+  BBO_CUDA(h, cudaEventRecord(h->ev0, s));
+  bbo::ffma_peak_kernel<<<h->sm_count, threads_per_sm, 0, s>>>(h->dbg_f.p, iters);
+  BBO_CUDA(h, cudaEventRecord(h->ev1, s));
+  BBO_CUDA(h, cudaGetLastError());
+  BBO_CUDA(h, cudaStreamSynchronize(s));
+  float ms = 0.f;
+  BBO_CUDA(h, cudaEventElapsedTime(&ms, h->ev0, h->ev1));
+  *tflops = (float)(2.0 * 16.0 * (double)iters * threads_per_sm * h->sm_count / (ms * 1e-3) / 1e12);
   return BBO_OK;
 }
 
@@ -727,7 +747,7 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
   FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr};
   int launches = 0;
   cudaError_t cuda_err = cudaSuccess;
-  rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, &launches, &cuda_err);
+  rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, 0, &launches, &cuda_err);
   if (rc != BBO_OK) return rc;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(fold_scores, n_configs, K, out_scores);
   if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return BBO_ERR_CUDA;

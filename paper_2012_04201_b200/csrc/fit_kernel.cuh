@@ -229,6 +229,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
   const int2 cf = a.fits[q];
   const int config = cf.x, fold = cf.y;
+  const uint32_t rng_config = (uint32_t)(config + a.config_base);  // index that keys the random streams
   const Config c = a.configs[config];
   const int H = c.hidden, d = a.d, CS = a.CS, TB = a.TB;
   const int dp = DPC ? DPC : a.dp;
@@ -263,7 +264,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     const float bound2 = __fsqrt_rn(__fdiv_rn(6.0f, (float)(H + CT)));
     const int n1 = d * H, n2 = H * CT;
     for (int blk = tid; blk < ((n1 + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, config, fold, 0u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 0u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const int idx = 4 * blk + w;
@@ -271,12 +272,12 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       }
     }
     for (int blk = tid; blk < ((H + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, config, fold, 1u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 1u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) { const int j = 4 * blk + w; if (j < H) v.W[L.ob1 + j] = glorot_value(word_of(r, w), bound1); }
     }
     for (int blk = tid; blk < ((n2 + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, config, fold, 2u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 2u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const int idx = 4 * blk + w;
@@ -284,7 +285,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       }
     }
     for (int blk = tid; blk < ((CT + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, config, fold, 3u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 3u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) { const int o = 4 * blk + w; if (o < CT) v.W[L.ob2 + o] = glorot_value(word_of(r, w), bound2); }
     }
@@ -313,7 +314,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     for (int j = 0; j < 8; ++j) v1[i][j] = 0.f;
 
   for (int e = 0; e < c.epochs; ++e) {
-    build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, vs, a.seed, config, fold, e, tid, nt);
+    build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, vs, a.seed, rng_config, fold, e, tid, nt);
     int buf = 0;
     {  // first sub-tile of the epoch
       const int Bs0 = n_tr < B ? n_tr : B, nb0 = Bs0 < TB ? Bs0 : TB;

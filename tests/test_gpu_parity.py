@@ -237,3 +237,49 @@ def test_error_codes(binding):
     caps = h.query_caps(64, 10)
     assert caps["max_hidden"] >= 200 and caps["max_classes"] >= 10
     h.close()
+
+
+def test_split_list_with_index_base_equals_unsplit_call(binding):
+    from paper_2012_04201_b200 import sharding
+    wl = W.workload("breast128", n_configs=11, epochs=5)
+    whole = gpu_eval(binding, wl, wl["configs"])
+    X = torch.from_numpy(wl["X"]).cuda()
+    y = torch.from_numpy(wl["y"]).cuda()
+    parts = []
+    for rank in range(3):
+        b, e = sharding.shard_bounds(11, rank, 3)
+        h = binding.MlpCv(config_index_base=b)
+        parts.append(h.eval(X, y, wl["task"], 5, wl["configs"][b:e], wl["seed"]).cpu().numpy())
+        h.close()
+    assert np.array_equal(np.concatenate(parts), whole["scores"])
+
+
+def test_register_fma_rate_is_near_the_nominal_peak(binding):
+    h = binding.MlpCv()
+    tf = h.debug_ffma_peak()
+    h.close()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    nominal = sms * 128 * 2 * 1.965e9 / 1e12
+    assert 0.6 * nominal < tf < 1.05 * nominal, tf
+
+
+def test_bench_workload_sampled_fits_match_oracle(binding):
+    """The launch configuration bench.py times (digits-shaped sweep, 4,000 fits, mixed widths
+    and batch sizes, 200 epochs), with a sample of whole fits recomputed by the checker."""
+    wl = W.workload("digits_sweep", seed=0, n_configs=800, epochs=200)
+    gpu = gpu_eval(binding, wl, wl["configs"])
+    assert np.all(np.isfinite(gpu["fold_scores"])) and gpu["fold_scores"].min() >= 0 and gpu["fold_scores"].max() <= 1
+    cfg = wl["configs"]
+    cost = cfg["hidden"].astype(np.float64)                      # cheap fits dominate the sample
+    order = np.argsort(cost)
+    pick = np.concatenate([order[:12], order[len(order) // 2: len(order) // 2 + 3], order[-1:]])
+    rng = np.random.default_rng(0)
+    fc = pick.astype(np.int32)
+    ff = rng.integers(0, 5, size=fc.size).astype(np.int32)
+    ref = oracle.cv_fits(wl["X"], wl["y"], wl["task"], 5, cfg, wl["seed"], fc, ff)["scores"]
+    got = gpu["fold_scores"][fc, ff].astype(np.float64)
+    print("[bench workload] sampled fits:", fc.size, "bit-equal:", int(np.sum(got == ref)))
+    assert np.mean(np.abs(got - ref) <= SCORE_ATOL) >= SCORE_FRACTION
+    m = gpu["fold_scores"].astype(np.float32)
+    mean = ((((m[:, 0] + m[:, 1]) + m[:, 2]) + m[:, 3]) + m[:, 4]) / np.float32(5)
+    assert np.array_equal(mean, gpu["scores"])
