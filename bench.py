@@ -146,25 +146,34 @@ def load_peaks():
 
 
 def oracle_sample_rate(wl, seconds_target=20.0, n_threads=0):
-    """Times the CPU checker, as it stands, on a sample of whole fits of this workload."""
+    """Times the CPU checker, as it stands, on a sample of this workload: one fit per host
+    thread (spread evenly over the step's fit list), each run for a reduced number of epochs
+    so that the sample takes about ``seconds_target`` seconds; the rate is scaled to whole fits
+    by the epoch ratio (cost is proportional to epochs)."""
     import oracle
 
     cores = oracle.num_procs() if n_threads <= 0 else n_threads
     cfg, K = wl["configs"], wl["n_folds"]
     n_fits = cfg.size * K
-    # about one full fit costs E*n_tr*(4dH+6HC) flops at roughly 1 GFLOP/s per core
     n, d = wl["X"].shape
+    epochs_full = int(cfg["epochs"][0])
+    # about one full fit costs E*n_tr*(4dH+6HC) flops at roughly 0.25 GFLOP/s per busy thread
     mean_flops = float((cfg["epochs"].astype(np.float64) * (n - n // K) * (4 * d + 60) * cfg["hidden"]).mean())
-    per_fit_s = mean_flops / 0.3e9  # measured: about 0.3 GFLOP/s per thread when all cores run
-    sample = int(max(cores, min(n_fits, round(seconds_target * cores / max(per_fit_s, 1e-3)))))
+    per_fit_s = mean_flops / 0.25e9
+    epochs_run = int(max(1, min(epochs_full, round(epochs_full * seconds_target / max(per_fit_s, 1e-3)))))
+    sample = int(min(n_fits, cores))
     idx = np.linspace(0, n_fits - 1, sample).astype(np.int64)
     fc, ff = (idx // K).astype(np.int32), (idx % K).astype(np.int32)
+    short = cfg.copy()
+    short["epochs"] = epochs_run
     t0 = time.perf_counter()
-    oracle.cv_fits(wl["X"], wl["y"], wl["task"], K, cfg, wl["seed"], fc, ff, n_threads=cores)
+    oracle.cv_fits(wl["X"], wl["y"], wl["task"], K, short, wl["seed"], fc, ff, n_threads=cores)
     dt = time.perf_counter() - t0
-    return dict(value=sample / dt, unit=UNIT, cores=cores, kind="oracle",
-                sample=f"{sample} whole fits (every {max(1, n_fits // sample)}th of the step's {n_fits}), "
-                       f"{dt:.1f} s wall on {cores} threads", seconds=dt, fits=sample)
+    fits_equiv = sample * epochs_run / float(epochs_full)
+    return dict(value=fits_equiv / dt, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{sample} fits (every {max(1, n_fits // sample)}th of the step's {n_fits}) for "
+                       f"{epochs_run} of {epochs_full} epochs, {dt:.1f} s wall on {cores} threads, "
+                       f"scaled to whole fits by the epoch ratio", seconds=dt, fits=fits_equiv)
 
 
 def run_reference(args, rank, world):
