@@ -191,15 +191,19 @@ struct FitBuffers {  // device scratch of one evaluation
   float* keep_theta;
 };
 
-// Groups the fits by padded hidden width, orders each group by descending cost estimate
-// E * n_train * (4dH + 6HC) + steps * 14 P, uploads the lists and launches one grid per group
-// (widest first; groups overlap on the side streams when there are any).
+// Orders the fits for launch.  Grids are dispatched in launch order, so the fits are first cut
+// into cost tiers (the costliest tenth, then 20 %, 30 %, 40 % of the fits) and, inside a tier,
+// grouped by padded hidden width (widest first) and sorted by descending cost: long fits start
+// early whatever their width, and the last launches hold only cheap fits, which keeps the tail
+// short.  Cost model (SM cycles, from phase timings): per optimizer step 8000 + 80 H fixed
+// (Adam, barriers, chain latencies) plus 2.9 H per row.  One grid per (tier, width) group, on
+// the side streams when there are any.
 int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk, const float* y, int n, int d,
                     int C, int K, int task, const bbo_mlp_config* configs, int n_configs, uint64_t seed,
                     int trace_steps, int maxB, int config_base, int* launches, cudaError_t* cuda_err) {
   *cuda_err = cudaSuccess;
   const int n_fits = n_configs * K;
-  struct Item { int Hs; double cost; int id; };
+  struct Item { int tier; int Hs; double cost; int id; };
   std::vector<Item> items((size_t)n_fits);
   for (int c = 0; c < n_configs; ++c) {
     const bbo_mlp_config& q = configs[c];
@@ -207,14 +211,23 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
       int vb, vs;
       bbo::fold_segment(n, K, f, &vb, &vs);
       const double n_tr = n - vs, B = std::min<double>(q.batch_size, n_tr);
-      const double P = (double)d * q.hidden + q.hidden + (double)q.hidden * C + C;
       const double steps = (double)q.epochs * std::ceil(n_tr / B);
-      items[(size_t)c * K + f] = {bbo::round_up(q.hidden, 8),
-                                  (double)q.epochs * n_tr * (4.0 * d * q.hidden + 6.0 * q.hidden * C) + steps * 14.0 * P,
-                                  c * K + f};
+      const double width = (double)q.hidden * (d + C) / 74.0;  // H for the 64-feature, 10-class shape
+      items[(size_t)c * K + f] = {0, bbo::round_up(q.hidden, 8),
+                                  steps * (8000.0 + 80.0 * width) + (double)q.epochs * n_tr * 2.9 * width, c * K + f};
+    }
+  }
+  {
+    std::vector<int> by_cost((size_t)n_fits);
+    for (int i = 0; i < n_fits; ++i) by_cost[i] = i;
+    std::stable_sort(by_cost.begin(), by_cost.end(), [&](int a, int b) { return items[a].cost > items[b].cost; });
+    for (int r = 0; r < n_fits; ++r) {
+      const double q = (double)r / n_fits;
+      items[by_cost[r]].tier = q < 0.10 ? 0 : (q < 0.30 ? 1 : (q < 0.60 ? 2 : 3));
     }
   }
   std::stable_sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
+    if (a.tier != b.tier) return a.tier < b.tier;
     return a.Hs != b.Hs ? a.Hs > b.Hs : a.cost > b.cost;
   });
   std::vector<int2> fits((size_t)n_fits);
@@ -224,7 +237,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
   std::vector<Group> groups;
   for (int i = 0; i < n_fits;) {
     int j = i;
-    while (j < n_fits && items[j].Hs == items[i].Hs) ++j;
+    while (j < n_fits && items[j].Hs == items[i].Hs && items[j].tier == items[i].tier) ++j;
     Group g{i, j - i, {}};
     const int rc = plan_bucket(env.smem_optin, n, d, C, K, items[i].Hs, maxB, trace_steps > 0, false, &g.plan);
     if (rc != BBO_OK) return rc;
