@@ -283,3 +283,24 @@ def test_bench_workload_sampled_fits_match_oracle(binding):
     m = gpu["fold_scores"].astype(np.float32)
     mean = ((((m[:, 0] + m[:, 1]) + m[:, 2]) + m[:, 3]) + m[:, 4]) / np.float32(5)
     assert np.array_equal(mean, gpu["scores"])
+
+
+def test_batched_studies_on_the_device_follow_the_checker(binding):
+    """Algorithm 1 with the device evaluation: several studies advance in lockstep, one call per
+    iteration; because scores are bit-equal to the checker's, the trajectories are identical."""
+    from paper_2012_04201_b200 import driver
+    wl = W.workload("iris8")
+    X = torch.from_numpy(wl["X"]).cuda()
+    y = torch.from_numpy(wl["y"]).cuda()
+    h = binding.MlpCv()
+
+    def make():
+        return [[driver.RandomSearch(10 + s, 12), driver.LocalPerturbation(20 + s, 12)] for s in range(3)]
+
+    dev = driver.run_studies(lambda c, sizes: h.eval(X, y, 0, 5, c, 0).cpu().numpy(), make(), n_step=3, n_batch=8)
+    ref = driver.run_studies(lambda c, sizes: oracle.cv_eval(wl["X"], wl["y"], 0, 5, c, 0)["scores"], make(),
+                             n_step=3, n_batch=8)
+    h.close()
+    for ld, lr in zip(dev, ref):
+        for (cd, sd), (cr, sr) in zip(ld, lr):
+            assert np.array_equal(cd, cr) and np.array_equal(sd, sr)
