@@ -126,11 +126,13 @@ int bbo_mlp_cv_debug_rng(bbo_mlp_cv* h, uint64_t seed, const uint32_t* counters,
                          uint32_t* out);
 int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* out);
 
-/* The Adam update needs one IEEE square root and one IEEE division per parameter per step;
- * the kernels use branch-free FMA-corrected versions inside a safe exponent range and the
- * IEEE routines outside it.  This export compares the two on the device.  mode 0: square root
- * of the `count` float bit patterns starting at `first`; mode 1: m / (sqrt(v) + eps) on
- * `count` pseudo-random operand triples keyed by `seed`.  host_out4: HOST [4] = number of
+/* The Adam update needs one IEEE square root and one IEEE division per parameter per step,
+ * the softmax one IEEE division per class and row; the kernels use branch-free FMA-corrected
+ * versions inside a safe exponent range and the IEEE routines outside it.  This export
+ * compares the two on the device.  mode 0: square root of the `count` float bit patterns
+ * starting at `first`; mode 1: m / (sqrt(v) + eps) on `count` pseudo-random operand triples
+ * keyed by `seed`; mode 2: softmax quotients exp(-t) / s, t in [0, 90), s in [1, 16], on
+ * `count` pseudo-random pairs.  host_out4: HOST [4] = number of
  * bit-level disagreements, number of cases taken by the fast path, and (for diagnosis) the
  * operand bits of one disagreement.                                                       */
 int bbo_mlp_cv_debug_fast_math(bbo_mlp_cv* h, int32_t mode, uint64_t seed, uint64_t first,

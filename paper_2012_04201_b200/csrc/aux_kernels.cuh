@@ -82,6 +82,16 @@ __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, 
       const float a = adam_denominator_fast(x, eps), b = __fadd_rn(__fsqrt_rn(x), eps);
       const float a2 = __fmul_rn(sqrt_fast_rn(fmaxf(__fmul_rn(x, 0x1p+96f), 0x1p-60f)), 0x1p-48f), b2 = __fsqrt_rn(x);
       if (__float_as_uint(a) != __float_as_uint(b) || (x != 0.f && __float_as_uint(a2) != __float_as_uint(b2))) { ++bad; out[2] = __float_as_uint(x); }
+    } else if (mode == 2) {  // softmax quotient: e = exp of a non-positive number, s in [1, 16]
+      const uint4 r = philox4x32_10(seed, 8u, (uint32_t)(i >> 32), 0u, 0u, (uint32_t)i);
+      const float e = spec_expf(-90.0f * (__uint2float_rn(r.x >> 8) * 0x1p-24f));
+      const float s = __fadd_rn(1.0f, __fmul_rn(15.0f, __uint2float_rn(r.y >> 8) * 0x1p-24f));
+      uint32_t safe = 1u;
+      const float q = softmax_ratio_fast(e, s, safe);
+      if (safe == 0u) continue;
+      ++safe_n;
+      const float ref = __fdiv_rn(e, s);
+      if (__float_as_uint(q) != __float_as_uint(ref)) { ++bad; out[2] = __float_as_uint(e); out[3] = __float_as_uint(s); }
     } else {
       const uint4 r = philox4x32_10(seed, 7u, (uint32_t)(i >> 32), 0u, 0u, (uint32_t)i);
       const float m = __uint_as_float(r.x);

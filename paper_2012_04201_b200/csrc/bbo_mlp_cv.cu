@@ -145,8 +145,8 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
   if (p.NT > bbo::kMaxFitThreads) return BBO_ERR_UNSUPPORTED;
   const size_t budget = (size_t)smem_optin - 256;  // static block scalars
   for (int TB = 32; TB >= 8; TB >>= 1) {
-    const size_t plain = bbo::fit_smem_bytes(d, p.dp, Hs, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, false);
-    const size_t lean = bbo::fit_smem_bytes(d, p.dp, Hs, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
+    const size_t plain = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, false);
+    const size_t lean = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
     if (lean > budget) continue;
     p.TB = TB;
     if (probe_only) {
@@ -562,7 +562,7 @@ int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* ou
 
 int bbo_mlp_cv_debug_fast_math(bbo_mlp_cv* h, int32_t mode, uint64_t seed, uint64_t first, uint64_t count,
                                uint64_t* host_out4) {
-  if (!h || !host_out4 || count < 1 || (mode != 0 && mode != 1)) return BBO_ERR_INVALID_ARG;
+  if (!h || !host_out4 || count < 1 || (mode < 0 || mode > 2)) return BBO_ERR_INVALID_ARG;
   DeviceGuard g(h->device);
   cudaStream_t s = h->stream;
   BBO_CUDA(h, h->dbg_u.reserve(8));

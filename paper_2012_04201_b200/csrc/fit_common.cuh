@@ -35,15 +35,19 @@ struct FitArgs {
 
 __host__ __device__ inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
-// Shared-memory layout of one fit (float offsets inside a parameter-sized block).
+// Shared-memory layout of one fit (float offsets inside a parameter-sized block).  W1 is
+// [d][Hs]; W2 is stored transposed, [C][Hs + 4] (class-major, so that the output layer reads
+// four consecutive hidden units of one class with one 16-byte load; the pitch of Hs + 4 keeps
+// the classes of one load on different banks).  Columns H..Hs+3 of W2 stay zero.
 struct Layout {
-  int Hs, oW1, ob1, oW2, ob2, PS, PT;
-  __host__ __device__ Layout(int d, int Hs_, int CS) {
+  int Hs, WP, oW1, ob1, oW2, ob2, PS, PT;
+  __host__ __device__ Layout(int d, int Hs_, int C, int CS) {
     Hs = Hs_;
+    WP = Hs + 4;           // pitch of a W2 class row, also of an A1 / delta1 row
     oW1 = 0;
     ob1 = d * Hs;
     oW2 = ob1 + Hs;
-    ob2 = oW2 + Hs * CS;   // W2 has Hs rows; rows H..Hs-1 stay zero
+    ob2 = oW2 + C * WP;
     PS = ob2 + CS;
     PT = PS - ob1;         // everything but W1
   }
@@ -61,12 +65,12 @@ constexpr int kSortBuckets = 2048;  // power of two
 __host__ __device__ inline size_t sort_scratch_bytes(int n) { return 8u * (size_t)round_up(n, 2) + 4u * kSortBuckets; }
 
 // Dynamic shared memory of one fit.  vreg: second moments of W1 live in registers.
-__host__ __device__ inline size_t fit_smem_bytes(int d, int dp, int Hs, int CS, int TB, int order_bytes,
+__host__ __device__ inline size_t fit_smem_bytes(int d, int dp, int Hs, int C, int CS, int TB, int order_bytes,
                                                  int loss_cap, int n_sort, bool vreg) {
-  const Layout L(d, Hs, CS);
+  const Layout L(d, Hs, C, CS);
   size_t bytes = 4u * (size_t)(2 * L.PS + (vreg ? L.PT : L.PS));
   bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + 8u * TB + 4u * (size_t)TB * CS;
-  const size_t xa = 8u * (size_t)TB * dp + 4u * (size_t)TB * Hs;
+  const size_t xa = 8u * (size_t)TB * dp + 4u * (size_t)TB * (Hs + 4);
   const size_t keys = sort_scratch_bytes(n_sort);
   return bytes + (xa > keys ? xa : keys);
 }

@@ -17,8 +17,9 @@
 // shared-memory instruction issue, not capacity, is what limits the register-tiled loops:
 //   stage   cp.async gather of the next sub-tile's rows, double buffered
 //   hidden  8x4 register tiles of A1 = relu(X W1 + b1), k ascending
-//   output  one lane per z2[b][o] (32/C rows per warp, two rows in flight per lane),
-//           j ascending, softmax and loss derivative with warp shuffles in the same lanes
+//   output  a lane pair per row, each lane half of the classes; W2 is kept class-major so one
+//           16-byte load feeds four steps of a chain; operands fetched one iteration ahead;
+//           softmax and loss derivative in the same lanes (two shuffles per scan)
 //   unit    one thread per hidden unit j: gW2[j][:], delta1[:, j] (in place over A1), gb1[j]
 //   gW1     8x8 register tiles that persist across sub-tiles, b ascending; the owner applies
 //           the L2 term and Adam to exactly its elements (second moments of W1 may stay in
@@ -31,6 +32,18 @@
 
 #include "device_math.cuh"
 #include "fit_common.cuh"
+
+// Optional phase timers (compile with -DBBO_PHASE_TIMERS): thread 0 accumulates clock64 deltas
+// per phase, as seen after the barrier that ends the phase, and block 0 of each launch prints
+// them.  Compiled out by default.
+#ifdef BBO_PHASE_TIMERS
+#include <cstdio>
+#define BBO_PHASE_BEGIN() long long ph_t_ = clock64()
+#define BBO_PHASE(i) do { if (tid == 0) { const long long t_ = clock64(); sh.phase[i] += t_ - ph_t_; ph_t_ = t_; } } while (0)
+#else
+#define BBO_PHASE_BEGIN() do { } while (0)
+#define BBO_PHASE(i) do { } while (0)
+#endif
 
 namespace bbo {
 
@@ -112,40 +125,71 @@ __device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L
       o.y = acc[i][1] > 0.f ? acc[i][1] : 0.f;
       o.z = acc[i][2] > 0.f ? acc[i][2] : 0.f;
       o.w = acc[i][3] > 0.f ? acc[i][3] : 0.f;
-      *reinterpret_cast<float4*>(v.A1 + (b0 + i) * Hs + j0) = o;
+      *reinterpret_cast<float4*>(v.A1 + (b0 + i) * L.WP + j0) = o;
     }
   }
 }
 
-// Logits of up to two rows per lane: z2[b][o] = b2[o] + sum_j A1[b][j] W2[j][o], j ascending.
-// Row b0 is valid when act0, row b1 when act1 (act1 implies act0).
-__device__ __forceinline__ void output_logits2(const FitView& v, const Layout& L, int CS, int Hs, int H, int o,
-                                               int b0, bool act0, int b1, bool act1, float& z0, float& z1) {
-  z0 = 0.f;
-  z1 = 0.f;
-  if (!act0) return;
-  const float bias = v.W[L.ob2 + o];
-  float acc0 = bias, acc1 = bias;
-  const float* r0 = v.A1 + b0 * Hs;
-  const float* r1 = v.A1 + (act1 ? b1 : b0) * Hs;
-  const float* wcol = v.W + L.oW2 + o;
+// Output layer.  A lane owns one row of the sub-tile and one half of the classes: classes
+// [0, QA) for the even lane of a pair, [QA, CT) for the odd lane, QA = ceil(CT / 2).  One
+// 16-byte load of the A1 row and one of each class row of W2 feed four steps of every chain:
+// z2[b][o] = b2[o] + sum_j A1[b][j] W2[j][o], j ascending.  (Shared-memory loads are what
+// bounds this phase, and this shape needs the fewest of them per multiply-add.)
+template <int CT>
+struct OutLane {
+  static constexpr int QA = (CT + 1) / 2, QB = CT - QA;
+  int half, o0, nq;  // this lane's classes are o0 .. o0 + nq - 1
+  __device__ __forceinline__ explicit OutLane(int lane) {
+    half = lane & 1;
+    o0 = half ? QA : 0;
+    nq = half ? QB : QA;
+  }
+  __device__ __forceinline__ int cls(int q) const { return q < nq ? o0 + q : o0 + (nq > 0 ? nq - 1 : -o0); }
+};
+
+template <int CT>
+__device__ __forceinline__ void output_logits(const FitView& v, const Layout& L, int H, const OutLane<CT>& ol, int row,
+                                              float (&z)[OutLane<CT>::QA]) {
+  constexpr int QA = OutLane<CT>::QA;
+  const float* wrow[QA];
+#pragma unroll
+  for (int q = 0; q < QA; ++q) {
+    const int o = ol.cls(q);  // lanes with fewer classes repeat their last one (result unused)
+    z[q] = v.W[L.ob2 + o];
+    wrow[q] = v.W + L.oW2 + o * L.WP;
+  }
+  const float* arow = v.A1 + row * L.WP;
+  // Few warps run this phase, so nothing else hides the load latency: the operands of the
+  // next four steps are fetched before the current four multiply-adds are issued.
   int j = 0;
+  float4 a_nx = *reinterpret_cast<const float4*>(arow);
+  float4 w_nx[QA];
+#pragma unroll
+  for (int q = 0; q < QA; ++q) w_nx[q] = *reinterpret_cast<const float4*>(wrow[q]);
+#pragma unroll 2
   for (; j + 4 <= H; j += 4) {
-    const float4 a0 = *reinterpret_cast<const float4*>(r0 + j);
-    const float4 a1 = *reinterpret_cast<const float4*>(r1 + j);
-    const float w0 = wcol[j * CS], w1 = wcol[(j + 1) * CS], w2 = wcol[(j + 2) * CS], w3 = wcol[(j + 3) * CS];
-    acc0 = __fmaf_rn(a0.x, w0, acc0); acc1 = __fmaf_rn(a1.x, w0, acc1);
-    acc0 = __fmaf_rn(a0.y, w1, acc0); acc1 = __fmaf_rn(a1.y, w1, acc1);
-    acc0 = __fmaf_rn(a0.z, w2, acc0); acc1 = __fmaf_rn(a1.z, w2, acc1);
-    acc0 = __fmaf_rn(a0.w, w3, acc0); acc1 = __fmaf_rn(a1.w, w3, acc1);
+    const float4 a = a_nx;
+    float4 w[QA];
+#pragma unroll
+    for (int q = 0; q < QA; ++q) w[q] = w_nx[q];
+    // rows are padded by four floats, so the read past the last step stays inside the row
+    a_nx = *reinterpret_cast<const float4*>(arow + j + 4);
+#pragma unroll
+    for (int q = 0; q < QA; ++q) w_nx[q] = *reinterpret_cast<const float4*>(wrow[q] + j + 4);
+#pragma unroll
+    for (int q = 0; q < QA; ++q) z[q] = __fmaf_rn(a.x, w[q].x, z[q]);
+#pragma unroll
+    for (int q = 0; q < QA; ++q) z[q] = __fmaf_rn(a.y, w[q].y, z[q]);
+#pragma unroll
+    for (int q = 0; q < QA; ++q) z[q] = __fmaf_rn(a.z, w[q].z, z[q]);
+#pragma unroll
+    for (int q = 0; q < QA; ++q) z[q] = __fmaf_rn(a.w, w[q].w, z[q]);
   }
   for (; j < H; ++j) {
-    const float w = wcol[j * CS];
-    acc0 = __fmaf_rn(r0[j], w, acc0);
-    acc1 = __fmaf_rn(r1[j], w, acc1);
+    const float a = arow[j];
+#pragma unroll
+    for (int q = 0; q < QA; ++q) z[q] = __fmaf_rn(a, wrow[q][j], z[q]);
   }
-  z0 = acc0;
-  z1 = acc1;
 }
 
 // Adam on one parameter with its gradient (L2 term already added for weights).
@@ -194,38 +238,79 @@ struct BlockShared {  // block-wide scalars
   int correct;
   float sq;
   float red[32];
+#ifdef BBO_PHASE_TIMERS
+  long long phase[12];
+#endif
 };
 
-// Softmax (or residual) of one row held across CT lanes starting at lane `obase`; returns this
-// lane's loss derivative.  All 32 lanes must call it.
+// Loss derivative of one row from the logits held by a lane pair, written to D2[row][:].
+// Classification: running maximum and softmax denominator are taken over the classes in
+// ascending order; the odd lane continues both scans from the even lane's result.  All 32 lanes
+// must call it; `active` gates the stores.
 template <int CT>
-__device__ __forceinline__ float row_delta(const FitView& v, int task, float z, float yv, int ocol, int obase,
-                                           bool active, float invB, bool want_loss, int loss_idx) {
+__device__ __forceinline__ void row_delta(const FitView& v, int task, int CS, const OutLane<CT>& ol,
+                                          const float (&z)[OutLane<CT>::QA], float yv, int row, bool active, float invB,
+                                          bool want_loss, int loss_idx) {
+  constexpr int QA = OutLane<CT>::QA;
   if (task == 0) {
     const int label = (int)yv;
-    float mx = __shfl_sync(0xffffffffu, z, obase);
+    // maximum: ascending scan with strict >, started by the even lane
+    float mx = z[0];
 #pragma unroll
-    for (int o = 1; o < CT; ++o) { const float t = __shfl_sync(0xffffffffu, z, obase + o); if (t > mx) mx = t; }
-    const float ex = spec_expf(__fsub_rn(z, mx));
-    float sum = 0.f;
+    for (int q = 1; q < QA; ++q) if (z[q] > mx) mx = z[q];
+    const float m_even = __shfl_sync(0xffffffffu, mx, (threadIdx.x & 31) & ~1);
+    if (ol.half) {
+      mx = m_even;
 #pragma unroll
-    for (int o = 0; o < CT; ++o) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, ex, obase + o));
-    const float pr = sum != sum ? sum : __fdiv_rn(ex, sum);  // NaN row: skip the library's special-case path
-    if (want_loss) {
-      const float zl = __shfl_sync(0xffffffffu, z, obase + (active ? label : 0));
-      if (active && ocol == 0) v.lossb[loss_idx] = __fsub_rn(logf(sum), __fsub_rn(zl, mx));
+      for (int q = 0; q < QA; ++q) if (q < ol.nq && z[q] > mx) mx = z[q];
     }
-    return __fmul_rn(__fsub_rn(pr, ocol == label ? 1.0f : 0.0f), invB);
+    mx = __shfl_sync(0xffffffffu, mx, (threadIdx.x & 31) | 1);
+    float ex[QA];
+#pragma unroll
+    for (int q = 0; q < QA; ++q) ex[q] = spec_expf(__fsub_rn(z[q], mx));
+    // denominator: ascending sum from zero, continued by the odd lane
+    float sum = 0.f;
+    if (!ol.half) {
+#pragma unroll
+      for (int q = 0; q < QA; ++q) sum = __fadd_rn(sum, ex[q]);
+    }
+    const float s_even = __shfl_sync(0xffffffffu, sum, (threadIdx.x & 31) & ~1);
+    if (ol.half) {
+      sum = s_even;
+#pragma unroll
+      for (int q = 0; q < QA; ++q) if (q < ol.nq) sum = __fadd_rn(sum, ex[q]);
+    }
+    sum = __shfl_sync(0xffffffffu, sum, (threadIdx.x & 31) | 1);
+    // probabilities: branch-free division first; the IEEE routine only where it cannot be certified
+    float pr[QA];
+    uint32_t safe = 1u;
+#pragma unroll
+    for (int q = 0; q < QA; ++q) pr[q] = softmax_ratio_fast(ex[q], sum, safe);
+    if (!safe) {
+#pragma unroll
+      for (int q = 0; q < QA; ++q) pr[q] = sum != sum ? sum : __fdiv_rn(ex[q], sum);  // NaN row: skip the library's special cases
+    }
+    float zl = 0.f;
+#pragma unroll
+    for (int q = 0; q < QA; ++q) {
+      const int o = ol.o0 + q;
+      if (active && q < ol.nq) v.D2[row * CS + o] = __fmul_rn(__fsub_rn(pr[q], o == label ? 1.0f : 0.0f), invB);
+      if (o == label) zl = z[q];
+    }
+    if (want_loss && active && label >= ol.o0 && label < ol.o0 + ol.nq)
+      v.lossb[loss_idx] = __fsub_rn(logf(sum), __fsub_rn(zl, mx));
+    return;
   }
-  const float r = __fsub_rn(z, yv);
-  if (want_loss && active) v.lossb[loss_idx] = __fmul_rn(__fmul_rn(0.5f, r), r);
-  return __fmul_rn(r, invB);
+  if (active && !ol.half) {
+    const float r = __fsub_rn(z[0], yv);
+    if (want_loss) v.lossb[loss_idx] = __fmul_rn(__fmul_rn(0.5f, r), r);
+    v.D2[row * CS] = __fmul_rn(r, invB);
+  }
 }
 
 // The whole fit.  CT: class count.  VR: second moments of W1 in registers.
 template <int CT, bool VR, int HSC, int DPC>
 __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, BlockShared& sh) {
-  constexpr int RW = 32 / CT;           // rows per warp in the output phase
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
   const int2 cf = a.fits[q];
   const int config = cf.x, fold = cf.y;
@@ -234,12 +319,16 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   const int H = c.hidden, d = a.d, CS = a.CS, TB = a.TB;
   const int dp = DPC ? DPC : a.dp;
   const int Hs = HSC ? HSC : a.Hs;
-  const Layout L(d, Hs, CS);
+  const Layout L(d, Hs, CT, CS);
   int vb, vs;
   fold_segment(a.n, a.K, fold, &vb, &vs);
   const int n_tr = a.n - vs;
   const int B = c.batch_size < n_tr ? c.batch_size : n_tr;
 
+#ifdef BBO_PHASE_TIMERS
+  if (tid < 12) sh.phase[tid] = 0;
+#endif
+  BBO_PHASE_BEGIN();
   FitView v;
   v.W = smem;
   v.M = v.W + L.PS;
@@ -281,7 +370,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const int idx = 4 * blk + w;
-        if (idx < n2) { const int j = idx / CT, o = idx - j * CT; v.W[L.oW2 + j * CS + o] = glorot_value(word_of(r, w), bound2); }
+        if (idx < n2) { const int j = idx / CT, o = idx - j * CT; v.W[L.oW2 + o * L.WP + j] = glorot_value(word_of(r, w), bound2); }
       }
     }
     for (int blk = tid; blk < ((CT + 3) >> 2); blk += nt) {
@@ -292,15 +381,18 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   }
   __syncthreads();
 
+  BBO_PHASE(0);
   // ---- thread roles ----
   const int KG = dp >> 3, JG8 = Hs >> 3;
   const bool has_tile = tid < KG * JG8;            // gW1 tile owner (host guarantees KG*JG8 <= nt)
   const int kg = has_tile ? tid / JG8 : 0, jg = has_tile ? tid - kg * JG8 : 0;
   const int k0 = kg << 3, jA = jg << 2, jB = (jg + JG8) << 2;
-  const bool unit_role = tid < H;                   // hidden unit tid: W2 row, b1, delta1 column
-  const bool o_role = tid < CT;                     // gb2 / b2 owner
-  const int orow = lane / CT, ocol = lane - orow * CT, obase = orow < RW ? orow * CT : 0;
-  const int rows_per_pass = n_warps * RW;
+  const bool unit_role = tid < H;                   // hidden unit tid: W2 column, b1, delta1 column
+  const int o_first = nt >= 64 ? nt - 32 : 0;       // gb2 / b2 owners sit in the last warp, away from the unit threads
+  const bool o_role = tid >= o_first && tid < o_first + CT;
+  const int oo = tid - o_first;
+  const OutLane<CT> ol(lane);                       // output phase: lane pair = one row, each lane half the classes
+  constexpr int QA = OutLane<CT>::QA;
 
   const float beta1 = c.beta1, beta2 = c.beta2, eps = c.eps;
   const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
@@ -315,6 +407,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 
   for (int e = 0; e < c.epochs; ++e) {
     build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, vs, a.seed, rng_config, fold, e, tid, nt);
+    BBO_PHASE(1);
     int buf = 0;
     {  // first sub-tile of the epoch
       const int Bs0 = n_tr < B ? n_tr : B, nb0 = Bs0 < TB ? Bs0 : TB;
@@ -338,13 +431,14 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         for (int j = 0; j < 8; ++j) g1[i][j] = 0.f;
       float g2[CT], w2[CT], gb1 = 0.f, gb2 = 0.f;
 #pragma unroll
-      for (int o = 0; o < CT; ++o) { g2[o] = 0.f; w2[o] = unit_role ? v.W[L.oW2 + tid * CS + o] : 0.f; }
+      for (int o = 0; o < CT; ++o) { g2[o] = 0.f; w2[o] = unit_role ? v.W[L.oW2 + o * L.WP + tid] : 0.f; }
 
       for (int t0 = 0; t0 < Bs; t0 += TB) {
         const int nb = (Bs - t0) < TB ? (Bs - t0) : TB;
         // rows of this sub-tile have landed; everyone is past the previous gW1 phase
         cp_async_wait_all();
         __syncthreads();
+        BBO_PHASE(2);
         const float* xs = v.Xs + buf * TB * dp;
         const float* ysb = v.ys + buf * TB;
         {  // prefetch the next sub-tile of this epoch into the other buffer
@@ -358,21 +452,18 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         }
         forward_hidden(v, L, xs, d, dp, Hs, nb, tid, nt);
         __syncthreads();
+        BBO_PHASE(3);
 
-        // ---- output layer, softmax / residual, loss derivative (lanes own logits) ----
-        for (int bw = warp * RW; bw < nb; bw += 2 * rows_per_pass) {
-          const int b0 = bw + orow, b1 = b0 + rows_per_pass;
-          const bool act0 = orow < RW && b0 < nb, act1 = orow < RW && b1 < nb;
-          float z0, z1;
-          output_logits2(v, L, CS, Hs, H, ocol, b0, act0, b1, act1, z0, z1);
-          const float d0 = row_delta<CT>(v, a.task, z0, act0 ? ysb[b0] : 0.f, ocol, obase, act0, invB, want_loss, t0 + b0);
-          if (act0) v.D2[b0 * CS + ocol] = d0;
-          if (bw + rows_per_pass < nb) {  // warp-uniform
-            const float d1 = row_delta<CT>(v, a.task, z1, act1 ? ysb[b1] : 0.f, ocol, obase, act1, invB, want_loss, t0 + b1);
-            if (act1) v.D2[b1 * CS + ocol] = d1;
-          }
+        // ---- output layer, softmax / residual, loss derivative (lane pairs own rows) ----
+        for (int r0 = warp * 16; r0 < nb; r0 += n_warps * 16) {  // warp-uniform
+          const int brow = r0 + (lane >> 1);
+          const bool act = brow < nb;
+          float z[QA];
+          output_logits<CT>(v, L, H, ol, act ? brow : nb - 1, z);
+          row_delta<CT>(v, a.task, CS, ol, z, act ? ysb[brow] : 0.f, brow, act, invB, want_loss, t0 + brow);
         }
         __syncthreads();
+        BBO_PHASE(4);
 
         // ---- hidden unit tid: gW2[tid][:], delta1[:, tid] in place over A1, gb1[tid]; b ascending ----
         if (unit_role) {
@@ -383,7 +474,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
             float a1r[4], dl[4][C4 * 4], acc[4];
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
-              a1r[r] = ap[(b + r) * Hs];
+              a1r[r] = ap[(b + r) * L.WP];
 #pragma unroll
               for (int o4 = 0; o4 < C4; ++o4) {
                 const float4 t = *reinterpret_cast<const float4*>(v.D2 + (b + r) * CS + 4 * o4);
@@ -402,12 +493,12 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
               const float d1 = a1r[r] > 0.f ? acc[r] : 0.f;
-              ap[(b + r) * Hs] = d1;
+              ap[(b + r) * L.WP] = d1;
               gb1 = __fadd_rn(gb1, d1);
             }
           }
           for (; b < nb; ++b) {
-            const float a1 = ap[b * Hs];
+            const float a1 = ap[b * L.WP];
             float acc = 0.f;
 #pragma unroll
             for (int o = 0; o < CT; ++o) {
@@ -416,12 +507,13 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
               acc = __fmaf_rn(dv, w2[o], acc);
             }
             const float d1 = a1 > 0.f ? acc : 0.f;
-            ap[b * Hs] = d1;
+            ap[b * L.WP] = d1;
             gb1 = __fadd_rn(gb1, d1);
           }
         }
-        if (o_role) for (int b = 0; b < nb; ++b) gb2 = __fadd_rn(gb2, v.D2[b * CS + tid]);
+        if (o_role) for (int b = 0; b < nb; ++b) gb2 = __fadd_rn(gb2, v.D2[b * CS + oo]);
         __syncthreads();
+        BBO_PHASE(5);
 
         // ---- gW1 tile: rows k0..k0+7, columns jA..jA+3 and jB..jB+3, b ascending ----
         if (has_tile) {
@@ -432,8 +524,8 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           for (int b = 0; b < nb; ++b) {
             const float4 x0 = *reinterpret_cast<const float4*>(xp + b * dp);
             const float4 x1 = *reinterpret_cast<const float4*>(xp + b * dp + 4);
-            const float4 dA = *reinterpret_cast<const float4*>(da + b * Hs);
-            const float4 dB = *reinterpret_cast<const float4*>(db + b * Hs);
+            const float4 dA = *reinterpret_cast<const float4*>(da + b * L.WP);
+            const float4 dB = *reinterpret_cast<const float4*>(db + b * L.WP);
             const float xk[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
             const float ds[8] = {dA.x, dA.y, dA.z, dA.w, dB.x, dB.y, dB.z, dB.w};
 #pragma unroll
@@ -443,8 +535,10 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           }
         }
         buf ^= 1;
+        BBO_PHASE(6);
       }
       __syncthreads();  // A1 / D2 / W reads of this step are done; step size is visible
+      BBO_PHASE(7);
 
       // ---- loss trace (debug): row losses in ascending order plus the L2 term ----
       if (want_loss) {
@@ -452,7 +546,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         for (int k = 0; k < d; ++k)
           for (int j = tid; j < H; j += nt) { const float w = v.W[L.oW1 + k * Hs + j]; sq = __fmaf_rn(w, w, sq); }
         for (int j = tid; j < H; j += nt)
-          for (int o = 0; o < CT; ++o) { const float w = v.W[L.oW2 + j * CS + o]; sq = __fmaf_rn(w, w, sq); }
+          for (int o = 0; o < CT; ++o) { const float w = v.W[L.oW2 + o * L.WP + j]; sq = __fmaf_rn(w, w, sq); }
         for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
         if (lane == 0) sh.red[warp] = sq;
         __syncthreads();
@@ -535,7 +629,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         float wu[CT + 1], mu[CT + 1], vu[CT + 1], gu[CT + 1], wold[CT + 1];
 #pragma unroll
         for (int o = 0; o < CT; ++o) {
-          const int off = L.oW2 + tid * CS + o;
+          const int off = L.oW2 + o * L.WP + tid;
           wu[o] = w2[o]; mu[o] = v.M[off]; vu[o] = v.V[off];
           gu[o] = __fmaf_rn(aB, w2[o], g2[o]);
         }
@@ -549,21 +643,23 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         }
 #pragma unroll
         for (int o = 0; o < CT; ++o) {
-          const int off = L.oW2 + tid * CS + o;
+          const int off = L.oW2 + o * L.WP + tid;
           v.W[off] = wu[o]; v.M[off] = mu[o]; v.V[off] = vu[o];
         }
         v.W[L.ob1 + tid] = wu[CT]; v.M[L.ob1 + tid] = mu[CT]; v.V[L.ob1 + tid] = vu[CT];
       }
       if (o_role) {
-        const int off = L.ob2 + tid;
+        const int off = L.ob2 + oo;
         adam_one(v.W[off], v.M[off], v.V[off], gb2, beta1, beta2, omb1, omb2, step, eps);
       }
       ++step_no;
+      BBO_PHASE(8);
       // the barrier at the top of the next sub-tile (or after the epoch) orders these writes
     }
     __syncthreads();
   }
 
+  BBO_PHASE(2);
   // ---- held-out score ----
   if (tid == 0) { sh.correct = 0; sh.sq = 0.f; }
   __syncthreads();
@@ -574,28 +670,28 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     __syncthreads();
     forward_hidden(v, L, v.Xs, d, dp, Hs, nb, tid, nt);
     __syncthreads();
-    for (int bw = warp * RW; bw < nb; bw += 2 * rows_per_pass) {
-      const int b0 = bw + orow, b1 = b0 + rows_per_pass;
-      const bool act0 = orow < RW && b0 < nb, act1 = orow < RW && b1 < nb;
-      float zz[2];
-      output_logits2(v, L, CS, Hs, H, ocol, b0, act0, b1, act1, zz[0], zz[1]);
+    for (int r0 = warp * 16; r0 < nb; r0 += n_warps * 16) {  // warp-uniform
+      const int brow = r0 + (lane >> 1);
+      const bool act = brow < nb;
+      float z[QA];
+      output_logits<CT>(v, L, H, ol, act ? brow : nb - 1, z);
+      if (a.task == 0) {
+        // prediction: ascending scan with strict >, started by the even lane, finished by the odd one
+        float best = z[0];
+        int besti = ol.o0;
 #pragma unroll
-      for (int cidx = 0; cidx < 2; ++cidx) {
-        const float z = zz[cidx];
-        const int b = cidx ? b1 : b0;
-        const bool act = cidx ? act1 : act0;
-        if (a.task == 0) {
-          float best = __shfl_sync(0xffffffffu, z, obase);
-          int besti = 0;
+        for (int q = 1; q < QA; ++q) if (!ol.half && z[q] > best) { best = z[q]; besti = q; }
+        const float b_even = __shfl_sync(0xffffffffu, best, lane & ~1);
+        const int i_even = __shfl_sync(0xffffffffu, besti, lane & ~1);
+        if (ol.half) {
+          best = b_even;
+          besti = i_even;
 #pragma unroll
-          for (int o = 1; o < CT; ++o) {
-            const float t = __shfl_sync(0xffffffffu, z, obase + o);
-            if (t > best) { best = t; besti = o; }
-          }
-          if (act && ocol == 0 && besti == (int)v.ys[b]) atomicAdd(&sh.correct, 1);
-        } else if (act) {
-          v.D2[b * CS] = __fsub_rn(z, v.ys[b]);
+          for (int q = 0; q < QA; ++q) if (q < ol.nq && z[q] > best) { best = z[q]; besti = ol.o0 + q; }
+          if (act && besti == (int)v.ys[brow]) atomicAdd(&sh.correct, 1);
         }
+      } else if (act && !ol.half) {
+        v.D2[brow * CS] = __fsub_rn(z[0], v.ys[brow]);
       }
     }
     __syncthreads();
@@ -616,11 +712,18 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     }
     a.fold_scores[(size_t)config * a.K + fold] = score;
   }
+  BBO_PHASE(9);
+#ifdef BBO_PHASE_TIMERS
+  if (tid == 0 && q == 0)
+    printf("PH Hs=%d H=%d B=%d nt=%d steps=%d | init %lld sort %lld wait %lld hidden %lld output %lld unit %lld gw1 %lld endbar %lld adam %lld score %lld\n",
+           Hs, H, B, nt, step_no, sh.phase[0], sh.phase[1], sh.phase[2], sh.phase[3], sh.phase[4], sh.phase[5], sh.phase[6],
+           sh.phase[7], sh.phase[8], sh.phase[9]);
+#endif
   if (a.keep_theta != nullptr && config == a.n_configs - 1 && fold == a.K - 1) {
     const int n1 = d * H, n2 = H * CT;
     for (int i = tid; i < n1; i += nt) a.keep_theta[i] = v.W[L.oW1 + (i / H) * Hs + (i % H)];
     for (int i = tid; i < H; i += nt) a.keep_theta[n1 + i] = v.W[L.ob1 + i];
-    for (int i = tid; i < n2; i += nt) a.keep_theta[n1 + H + i] = v.W[L.oW2 + (i / CT) * CS + (i % CT)];
+    for (int i = tid; i < n2; i += nt) a.keep_theta[n1 + H + i] = v.W[L.oW2 + (i % CT) * L.WP + (i / CT)];
     for (int i = tid; i < CT; i += nt) a.keep_theta[n1 + H + n2 + i] = v.W[L.ob2 + i];
   }
 }

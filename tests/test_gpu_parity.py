@@ -101,6 +101,9 @@ def test_branch_free_sqrt_and_division_equal_ieee(binding):
         assert out[0] == 0, out
         total_safe += int(out[1])
     assert total_safe > 5e7
+    # softmax quotients: exponentials of non-positive numbers over denominators in [1, 16]
+    out = h.debug_fast_math(2, seed=3, count=2**30)
+    assert out[0] == 0 and out[1] > 1.0e9, out
     h.close()
 
 
