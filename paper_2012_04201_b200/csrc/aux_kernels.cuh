@@ -76,7 +76,7 @@ __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, 
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < count; i += (uint64_t)gridDim.x * blockDim.x) {
     if (mode == 0) {
       const float x = __uint_as_float((uint32_t)(first + i));
-      if (__float_as_uint(x) >= kVHi) continue;
+      if (!(x < 0x1p+30f)) continue;
       ++safe_n;
       const float eps = 0x1p-30f;
       const float a = adam_denominator_fast(x, eps), b = __fadd_rn(__fsqrt_rn(x), eps);
@@ -97,9 +97,9 @@ __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, 
       const float m = __uint_as_float(r.x);
       const float vv = __uint_as_float(r.y & 0x7FFFFFFFu);
       const float eps = __uint_as_float((r.z & 0x007FFFFFu) | ((20u + (r.w % 170u)) << 23));  // 2^-107 .. 2^62
-      uint32_t safe = adam_eps_safe(eps);
-      const float q = adam_ratio_fast(m, vv, eps, safe);
-      if (safe == 0u) continue;
+      AdamCert cert;
+      const float q = adam_ratio_fast(m, vv, eps, cert);
+      if ((adam_eps_safe(eps) & cert.ok()) == 0u) continue;
       ++safe_n;
       const float ref = adam_ratio_ieee(m, vv, eps);
       if (__float_as_uint(q) != __float_as_uint(ref)) { ++bad; out[2] = __float_as_uint(m); out[3] = __float_as_uint(vv); }

@@ -208,14 +208,14 @@ template <int N>
 __device__ __forceinline__ uint32_t adam_group_fast(float (&th)[N], float (&m)[N], float (&vv)[N], const float (&g)[N],
                                                     float beta1, float beta2, float omb1, float omb2, float step,
                                                     float eps, uint32_t eps_safe) {
-  uint32_t safe = eps_safe;
+  AdamCert cert;
 #pragma unroll
   for (int e = 0; e < N; ++e) {
     m[e] = __fmaf_rn(beta1, m[e], __fmul_rn(omb1, g[e]));
     vv[e] = __fmaf_rn(beta2, vv[e], __fmul_rn(__fmul_rn(omb2, g[e]), g[e]));
-    th[e] = __fsub_rn(th[e], __fmul_rn(step, adam_ratio_fast(m[e], vv[e], eps, safe)));
+    th[e] = __fsub_rn(th[e], __fmul_rn(step, adam_ratio_fast(m[e], vv[e], eps, cert)));
   }
-  return safe;
+  return eps_safe & cert.ok();
 }
 
 // Second pass for a group the first pass could not certify: IEEE square root and division.
