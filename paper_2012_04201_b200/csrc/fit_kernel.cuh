@@ -233,6 +233,25 @@ __device__ __forceinline__ void adam_params_ieee(float (&th)[N], const float (&m
   }
 }
 
+// Operands of one row of the W1 gradient tile: x[b][k0..k0+7] and delta1[b][jA..jA+3, jB..jB+3].
+struct GradOperands {
+  float4 x0, x1, dA, dB;
+  __device__ __forceinline__ void load(const float* xp, const float* da, const float* db, int b, int dp, int wp) {
+    x0 = *reinterpret_cast<const float4*>(xp + b * dp);
+    x1 = *reinterpret_cast<const float4*>(xp + b * dp + 4);
+    dA = *reinterpret_cast<const float4*>(da + b * wp);
+    dB = *reinterpret_cast<const float4*>(db + b * wp);
+  }
+  __device__ __forceinline__ void accumulate(float (&g1)[8][8]) const {
+    const float xk[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+    const float ds[8] = {dA.x, dA.y, dA.z, dA.w, dB.x, dB.y, dB.z, dB.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) g1[i][j] = __fmaf_rn(xk[i], ds[j], g1[i][j]);
+  }
+};
+
 struct BlockShared {  // block-wide scalars
   float step[2];  // Adam step size, indexed by step parity (writer runs ahead of readers)
   int correct;
@@ -517,22 +536,22 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 
         // ---- gW1 tile: rows k0..k0+7, columns jA..jA+3 and jB..jB+3, b ascending ----
         if (has_tile) {
+          // Two operand sets in flight: the loads of row b + 1 are issued before the multiply-adds
+          // of row b, so a warp does not sit out the shared-memory latency once per row.
           const float* xp = xs + k0;
           const float* da = v.A1 + jA;
           const float* db = v.A1 + jB;
-#pragma unroll 2
-          for (int b = 0; b < nb; ++b) {
-            const float4 x0 = *reinterpret_cast<const float4*>(xp + b * dp);
-            const float4 x1 = *reinterpret_cast<const float4*>(xp + b * dp + 4);
-            const float4 dA = *reinterpret_cast<const float4*>(da + b * L.WP);
-            const float4 dB = *reinterpret_cast<const float4*>(db + b * L.WP);
-            const float xk[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-            const float ds[8] = {dA.x, dA.y, dA.z, dA.w, dB.x, dB.y, dB.z, dB.w};
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-#pragma unroll
-              for (int j = 0; j < 8; ++j) g1[i][j] = __fmaf_rn(xk[i], ds[j], g1[i][j]);
+          GradOperands opA, opB;
+          opA.load(xp, da, db, 0, dp, L.WP);
+          int b = 0;
+#pragma unroll 1
+          for (; b + 2 <= nb; b += 2) {
+            opB.load(xp, da, db, b + 1, dp, L.WP);
+            opA.accumulate(g1);
+            opA.load(xp, da, db, b + 2 < nb ? b + 2 : b, dp, L.WP);
+            opB.accumulate(g1);
           }
+          if (b < nb) opA.accumulate(g1);
         }
         buf ^= 1;
         BBO_PHASE(6);
