@@ -20,6 +20,8 @@ _LIB = os.path.join(_HERE, "libmlp_cv_oracle.so")
 MODE_F32 = 0
 MODE_F64 = 1
 STREAM_FOLD, STREAM_INIT, STREAM_PERM = 1, 2, 3
+SOLVER_ADAM, SOLVER_SGD = 0, 1
+METRIC_DEFAULT, METRIC_ALT = 0, 1   # accuracy / -MSE, or -NLL / -MAE
 
 CONFIG_DTYPE = np.dtype(
     [("hidden", "<i4"), ("batch_size", "<i4"), ("epochs", "<i4"), ("alpha", "<f4"),
@@ -76,6 +78,12 @@ def lib():
         L.oracle_mlp_cv_eval.argtypes = [i32, vp, vp, i64, i32, i32, i32, vp, i32, u64, i32, i32, i32,
                                          vp, vp, vp]
         L.oracle_mlp_cv_eval.restype = ctypes.c_int
+        L.oracle_mlp_cv_fits_ex.argtypes = L.oracle_mlp_cv_fits.argtypes + [i32, i32]
+        L.oracle_mlp_cv_fits_ex.restype = ctypes.c_int
+        L.oracle_mlp_cv_eval_ex.argtypes = L.oracle_mlp_cv_eval.argtypes + [i32, i32]
+        L.oracle_mlp_cv_eval_ex.restype = ctypes.c_int
+        L.oracle_sgd_steps.argtypes = [i32, i64, i32, f64, f64, vp, vp, vp]
+        L.oracle_sgd_steps.restype = None
         L.oracle_num_procs.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -171,6 +179,15 @@ def adam_steps(mode, theta, m, v, grads, lr, beta1, beta2, eps):
     return theta, m, v
 
 
+def sgd_steps(mode, theta, vel, grads, lr, momentum):
+    """n momentum-SGD updates with the given gradients [n, P]; returns (theta, velocity)."""
+    theta = np.array(theta, np.float64)
+    vel = np.array(vel, np.float64)
+    grads = np.ascontiguousarray(grads, np.float64).reshape(-1, theta.size)
+    lib().oracle_sgd_steps(mode, theta.size, grads.shape[0], lr, momentum, _p(theta), _p(vel), _p(grads))
+    return theta, vel
+
+
 def _prep(X, y, configs):
     X = np.ascontiguousarray(X, np.float32)
     y = np.ascontiguousarray(y, np.float32)
@@ -180,8 +197,11 @@ def _prep(X, y, configs):
 
 
 def cv_fits(X, y, task, n_folds, configs, seed, fit_config, fit_fold, mode=MODE_F32, n_classes=0,
-            trace_steps=0, n_threads=0, want_theta=False):
-    """Run the listed (config, fold) fits.  Returns dict(scores, trace, theta)."""
+            trace_steps=0, n_threads=0, want_theta=False, solver=SOLVER_ADAM, metric=METRIC_DEFAULT):
+    """Run the listed (config, fold) fits.  Returns dict(scores, trace, theta).
+
+    solver: SOLVER_ADAM or SOLVER_SGD (Nesterov momentum = the configuration's beta1);
+    metric: METRIC_DEFAULT (accuracy / -MSE) or METRIC_ALT (-NLL / -MAE)."""
     X, y, configs = _prep(X, y, configs)
     n, d = X.shape
     fc = np.ascontiguousarray(fit_config, np.int32)
@@ -192,15 +212,16 @@ def cv_fits(X, y, task, n_folds, configs, seed, fit_config, fit_fold, mode=MODE_
     if want_theta:
         C = 1 if task == 1 else (n_classes or int(y.max()) + 1)
         theta = np.zeros(param_count(d, int(configs["hidden"][fc[-1]]), C), np.float64)
-    rc = lib().oracle_mlp_cv_fits(mode, _p(X), _p(y), n, d, task, n_folds, _p(configs), configs.size, seed,
-                                  n_classes, _p(fc), _p(ff), fc.size, trace_steps, n_threads, _p(scores),
-                                  _p(trace), _p(theta))
+    rc = lib().oracle_mlp_cv_fits_ex(mode, _p(X), _p(y), n, d, task, n_folds, _p(configs), configs.size, seed,
+                                     n_classes, _p(fc), _p(ff), fc.size, trace_steps, n_threads, _p(scores),
+                                     _p(trace), _p(theta), solver, metric)
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return dict(scores=scores, trace=trace, theta=theta)
 
 
-def cv_eval(X, y, task, n_folds, configs, seed, mode=MODE_F32, n_classes=0, trace_steps=0, n_threads=0):
+def cv_eval(X, y, task, n_folds, configs, seed, mode=MODE_F32, n_classes=0, trace_steps=0, n_threads=0,
+            solver=SOLVER_ADAM, metric=METRIC_DEFAULT):
     """scores = evaluate(params_list).  Returns dict(scores, fold_scores, trace)."""
     X, y, configs = _prep(X, y, configs)
     n, d = X.shape
@@ -208,8 +229,8 @@ def cv_eval(X, y, task, n_folds, configs, seed, mode=MODE_F32, n_classes=0, trac
     scores = np.zeros(nc, np.float64)
     fold_scores = np.zeros((nc, n_folds), np.float64)
     trace = np.zeros((nc * n_folds, trace_steps), np.float64) if trace_steps else None
-    rc = lib().oracle_mlp_cv_eval(mode, _p(X), _p(y), n, d, task, n_folds, _p(configs), nc, seed, n_classes,
-                                  trace_steps, n_threads, _p(scores), _p(fold_scores), _p(trace))
+    rc = lib().oracle_mlp_cv_eval_ex(mode, _p(X), _p(y), n, d, task, n_folds, _p(configs), nc, seed, n_classes,
+                                     trace_steps, n_threads, _p(scores), _p(fold_scores), _p(trace), solver, metric)
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return dict(scores=scores, fold_scores=fold_scores, trace=trace)

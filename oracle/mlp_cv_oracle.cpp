@@ -273,10 +273,30 @@ struct Adam {
   }
 };
 
+// Stochastic gradient descent with Nesterov momentum (the paper's Table 1 lists MLP-sgd beside
+// MLP-adam; this is the update of the scikit-learn solver it names, constant learning rate):
+// velocity = momentum * velocity - lr * g; theta += momentum * velocity - lr * g, the second
+// expression taken with the new velocity.  lr * g is rounded once and used in both; each of the
+// two expressions is one fused multiply-add.
+template <typename T>
+struct Sgd {
+  T lr, momentum;
+  void update(int64_t P, T* th, T* vel, const T* g) {
+    for (int64_t i = 0; i < P; ++i) {
+      const T t = lr * g[i];
+      vel[i] = Fn<T>::fma_(momentum, vel[i], -t);
+      th[i] = th[i] + Fn<T>::fma_(momentum, vel[i], -t);
+    }
+  }
+};
+
+enum : int32_t { SOLVER_ADAM = 0, SOLVER_SGD = 1 };
+enum : int32_t { METRIC_DEFAULT = 0, METRIC_ALT = 1 };  // accuracy / -MSE, or -NLL / -MAE (Table 1: nll, mae)
+
 // Held-out score of one fit: accuracy (prediction = lowest index attaining the maximum
 // under strict >, so a NaN never wins) or negative mean squared error (NaN -> -inf).
 template <typename T>
-T score_rows(const Shape& s, int32_t task, const T* th, const float* X, const float* y,
+T score_rows(const Shape& s, int32_t task, int32_t metric, const T* th, const float* X, const float* y,
              const int32_t* rows, int32_t n_rows) {
   std::vector<T> x((size_t)s.d), z1((size_t)s.H), a1((size_t)s.H), z2((size_t)s.C);
   int32_t correct = 0;
@@ -285,16 +305,28 @@ T score_rows(const Shape& s, int32_t task, const T* th, const float* X, const fl
     const float* xr = X + (int64_t)rows[i] * s.d;
     for (int32_t k = 0; k < s.d; ++k) x[k] = (T)xr[k];
     forward_row(s, th, x.data(), z1.data(), a1.data(), z2.data());
-    if (task == 0) {
+    if (task == 0 && metric == METRIC_ALT) {
+      // negative log-likelihood of the true class under the softmax (same max-subtraction,
+      // exponential and ascending denominator as in training), summed over rows in order
+      const int32_t label = (int32_t)y[rows[i]];
+      T mx = z2[0];
+      for (int32_t o = 1; o < s.C; ++o) if (z2[o] > mx) mx = z2[o];
+      T sum = (T)0;
+      for (int32_t o = 0; o < s.C; ++o) sum = sum + Fn<T>::exp_(z2[o] - mx);
+      sq = sq + (Fn<T>::log_(sum) - (z2[label] - mx));
+    } else if (task == 0) {
       int32_t best = 0;
       for (int32_t o = 1; o < s.C; ++o) if (z2[o] > z2[best]) best = o;
       if (best == (int32_t)y[rows[i]]) ++correct;
+    } else if (metric == METRIC_ALT) {
+      T r = z2[0] - (T)y[rows[i]];
+      sq = sq + (r < (T)0 ? -r : r);
     } else {
       T r = z2[0] - (T)y[rows[i]];
       sq = Fn<T>::fma_(r, r, sq);
     }
   }
-  if (task == 0) return (T)correct / (T)n_rows;
+  if (task == 0 && metric == METRIC_DEFAULT) return (T)correct / (T)n_rows;
   T s_ = -(sq / (T)n_rows);
   if (s_ != s_) s_ = -std::numeric_limits<T>::infinity();
   return s_;
@@ -306,7 +338,8 @@ T score_rows(const Shape& s, int32_t task, const T* th, const float* X, const fl
 template <typename T>
 double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, int32_t task,
                int32_t K, const Config& cf, uint32_t config, uint32_t fold, uint64_t seed,
-               const std::vector<int32_t>& pi, int32_t trace_steps, double* trace, double* theta_out) {
+               const std::vector<int32_t>& pi, int32_t trace_steps, double* trace, double* theta_out,
+               int32_t solver = SOLVER_ADAM, int32_t metric = METRIC_DEFAULT) {
   int64_t vb, vs;
   fold_segment(n, K, (int32_t)fold, &vb, &vs);
   std::vector<int32_t> val(pi.begin() + vb, pi.begin() + vb + vs), train;
@@ -319,6 +352,7 @@ double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, 
   std::vector<T> th((size_t)P), m((size_t)P, (T)0), v((size_t)P, (T)0), g((size_t)P);
   init_params<T>(s, seed, config, fold, th.data());
   Adam<T> adam{(T)cf.lr, (T)cf.beta1, (T)cf.beta2, (T)cf.eps};
+  Sgd<T> sgd{(T)cf.lr, (T)cf.beta1};  // beta1 doubles as the momentum
   std::vector<T> xb((size_t)B * d), yb((size_t)B);
   std::vector<int32_t> sigma;
   for (int32_t i = 0; i < trace_steps; ++i) if (trace) trace[i] = std::numeric_limits<double>::quiet_NaN();
@@ -335,12 +369,13 @@ double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, 
       const bool want = trace && step_no < trace_steps;
       T loss = loss_and_grad<T>(s, task, (T)cf.alpha, th.data(), xb.data(), yb.data(), Bs, g.data(), want);
       if (want) trace[step_no] = (double)loss;
-      adam.update(P, th.data(), m.data(), v.data(), g.data());
+      if (solver == SOLVER_SGD) sgd.update(P, th.data(), m.data(), g.data());
+      else adam.update(P, th.data(), m.data(), v.data(), g.data());
       ++step_no;
     }
   }
   if (theta_out) for (int64_t i = 0; i < P; ++i) theta_out[i] = (double)th[i];
-  return (double)score_rows<T>(s, task, th.data(), X, y, val.data(), (int32_t)val.size());
+  return (double)score_rows<T>(s, task, metric, th.data(), X, y, val.data(), (int32_t)val.size());
 }
 
 int validate(const float* X, const float* y, int64_t n, int32_t d, int32_t task, int32_t K,
@@ -477,11 +512,14 @@ void oracle_adam_steps(int32_t mode, int64_t P, int32_t n_steps, double lr, doub
 //   fit_config[n_fits], fit_fold[n_fits]: which fits to run (config index into configs[]).
 //   fit_scores[n_fits]; loss_trace[n_fits*trace_steps] (or null); theta_out: parameters of
 //   the LAST listed fit (or null).  n_threads <= 0: all cores; threads split fits only.
-int oracle_mlp_cv_fits(int32_t mode, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
-                       int32_t n_folds, const void* configs, int32_t n_configs, uint64_t seed,
-                       int32_t n_classes, const int32_t* fit_config, const int32_t* fit_fold, int32_t n_fits,
-                       int32_t trace_steps, int32_t n_threads, double* fit_scores, double* loss_trace,
-                       double* theta_out) {
+// solver: 0 Adam, 1 SGD with Nesterov momentum (momentum = the configuration's beta1).
+// metric: 0 accuracy / -MSE, 1 -NLL / -MAE.
+int oracle_mlp_cv_fits_ex(int32_t mode, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
+                          int32_t n_folds, const void* configs, int32_t n_configs, uint64_t seed,
+                          int32_t n_classes, const int32_t* fit_config, const int32_t* fit_fold, int32_t n_fits,
+                          int32_t trace_steps, int32_t n_threads, double* fit_scores, double* loss_trace,
+                          double* theta_out, int32_t solver, int32_t metric) {
+  if (solver < 0 || solver > 1 || metric < 0 || metric > 1) return -1;
   const Config* cfg = (const Config*)configs;
   if (validate(X, y, n, d, task, n_folds, cfg, n_configs) != 0) return -1;
   const int32_t C = derive_classes(y, n, task, n_classes);
@@ -499,24 +537,34 @@ int oracle_mlp_cv_fits(int32_t mode, const float* X, const float* y, int64_t n, 
     double* tho = (theta_out && i == n_fits - 1) ? theta_out : nullptr;
     const Config& cf = cfg[fit_config[i]];
     fit_scores[i] = mode == 1
-        ? run_fit<double>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho)
-        : run_fit<float>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho);
+        ? run_fit<double>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho, solver, metric)
+        : run_fit<float>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho, solver, metric);
   }
   return 0;
 }
 
+int oracle_mlp_cv_fits(int32_t mode, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
+                       int32_t n_folds, const void* configs, int32_t n_configs, uint64_t seed,
+                       int32_t n_classes, const int32_t* fit_config, const int32_t* fit_fold, int32_t n_fits,
+                       int32_t trace_steps, int32_t n_threads, double* fit_scores, double* loss_trace,
+                       double* theta_out) {
+  return oracle_mlp_cv_fits_ex(mode, X, y, n, d, task, n_folds, configs, n_configs, seed, n_classes, fit_config,
+                               fit_fold, n_fits, trace_steps, n_threads, fit_scores, loss_trace, theta_out, 0, 0);
+}
+
 // scores = evaluate(params_list): every config, every fold, mean over folds (ascending fold,
 // in the mode's precision).  fold_scores[n_configs*n_folds] and loss_trace may be null.
-int oracle_mlp_cv_eval(int32_t mode, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
-                       int32_t n_folds, const void* configs, int32_t n_configs, uint64_t seed,
-                       int32_t n_classes, int32_t trace_steps, int32_t n_threads, double* out_scores,
-                       double* fold_scores, double* loss_trace) {
+int oracle_mlp_cv_eval_ex(int32_t mode, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
+                          int32_t n_folds, const void* configs, int32_t n_configs, uint64_t seed,
+                          int32_t n_classes, int32_t trace_steps, int32_t n_threads, double* out_scores,
+                          double* fold_scores, double* loss_trace, int32_t solver, int32_t metric) {
   const int32_t n_fits = n_configs * n_folds;
   std::vector<int32_t> fc((size_t)n_fits), ff((size_t)n_fits);
   for (int32_t i = 0; i < n_fits; ++i) { fc[i] = i / n_folds; ff[i] = i % n_folds; }
   std::vector<double> fs((size_t)n_fits);
-  int rc = oracle_mlp_cv_fits(mode, X, y, n, d, task, n_folds, configs, n_configs, seed, n_classes, fc.data(),
-                              ff.data(), n_fits, trace_steps, n_threads, fs.data(), loss_trace, nullptr);
+  int rc = oracle_mlp_cv_fits_ex(mode, X, y, n, d, task, n_folds, configs, n_configs, seed, n_classes, fc.data(),
+                                 ff.data(), n_fits, trace_steps, n_threads, fs.data(), loss_trace, nullptr, solver,
+                                 metric);
   if (rc != 0) return rc;
   for (int32_t c = 0; c < n_configs; ++c) {
     if (mode == 1) {
@@ -531,6 +579,31 @@ int oracle_mlp_cv_eval(int32_t mode, const float* X, const float* y, int64_t n, 
   }
   if (fold_scores) std::copy(fs.begin(), fs.end(), fold_scores);
   return 0;
+}
+
+int oracle_mlp_cv_eval(int32_t mode, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
+                       int32_t n_folds, const void* configs, int32_t n_configs, uint64_t seed,
+                       int32_t n_classes, int32_t trace_steps, int32_t n_threads, double* out_scores,
+                       double* fold_scores, double* loss_trace) {
+  return oracle_mlp_cv_eval_ex(mode, X, y, n, d, task, n_folds, configs, n_configs, seed, n_classes, trace_steps,
+                               n_threads, out_scores, fold_scores, loss_trace, 0, 0);
+}
+
+// n_steps momentum-SGD updates on P parameters with caller-supplied gradients grads[n_steps][P].
+void oracle_sgd_steps(int32_t mode, int64_t P, int32_t n_steps, double lr, double momentum, double* theta,
+                      double* vel, const double* grads) {
+  if (mode == 1) {
+    Sgd<double> a{lr, momentum};
+    for (int32_t s = 0; s < n_steps; ++s) a.update(P, theta, vel, grads + (int64_t)s * P);
+    return;
+  }
+  std::vector<float> th(theta, theta + P), vv(vel, vel + P), g((size_t)P);
+  Sgd<float> a{(float)lr, (float)momentum};
+  for (int32_t s = 0; s < n_steps; ++s) {
+    for (int64_t i = 0; i < P; ++i) g[i] = (float)grads[(int64_t)s * P + i];
+    a.update(P, th.data(), vv.data(), g.data());
+  }
+  for (int64_t i = 0; i < P; ++i) { theta[i] = th[i]; vel[i] = vv[i]; }
 }
 
 int oracle_num_procs(void) {

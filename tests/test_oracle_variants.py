@@ -1,0 +1,139 @@
+"""Pins for the checker's variants: the SGD solver (paper Table 1: MLP-sgd) and the nll / mae
+metrics (paper Table 1), each against something other than the checker itself."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2012_04201_b200 import workloads as W
+from test_oracle_fit import one_config, unpack
+
+
+def test_sgd_first_step_closed_form_zero_lr_and_zero_momentum():
+    rng = np.random.default_rng(0)
+    P = 40
+    th0 = rng.normal(size=P)
+    g = rng.normal(size=(1, P))
+    lr, mom = 0.03, 0.9
+    th, vel = oracle.sgd_steps(1, th0, np.zeros(P), g, lr, mom)
+    # from zero velocity: velocity = -lr g, Nesterov look-ahead moves by -(1 + momentum) lr g
+    np.testing.assert_allclose(vel, -lr * g[0], rtol=1e-15)
+    np.testing.assert_allclose(th, th0 - (1 + mom) * lr * g[0], rtol=1e-14)
+    # lr = 0 leaves parameters bit-unchanged over many steps (float mode)
+    th32 = th0.astype(np.float32).astype(np.float64)
+    th, vel = oracle.sgd_steps(0, th32, np.zeros(P), rng.normal(size=(20, P)), 0.0, mom)
+    assert np.array_equal(th, th32) and not vel.any()
+    # momentum = 0 is plain gradient descent
+    gs = rng.normal(size=(7, P))
+    th, _ = oracle.sgd_steps(1, th0, np.zeros(P), gs, lr, 0.0)
+    np.testing.assert_allclose(th, th0 - lr * gs.sum(0), rtol=1e-13, atol=1e-15)
+
+
+def test_sgd_matches_torch_nesterov_over_many_steps():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(1)
+    P, n = 30, 40
+    th0 = rng.normal(size=P)
+    grads = rng.normal(size=(n, P))
+    lr, mom = 0.02, 0.8
+    got, _ = oracle.sgd_steps(1, th0, np.zeros(P), grads, lr, mom)
+    # torch's SGD keeps buf = mom buf + g and steps by lr (g + mom buf): the same iteration with
+    # velocity = -lr buf
+    p = torch.tensor(th0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([p], lr=lr, momentum=mom, nesterov=True)
+    for t in range(n):
+        p.grad = torch.tensor(grads[t])
+        opt.step()
+    np.testing.assert_allclose(got, p.detach().numpy(), rtol=1e-11, atol=1e-13)
+
+
+@pytest.mark.parametrize("task,C", [(0, 3), (1, 1)])
+def test_sgd_five_steps_match_scikit_learn(task, C):
+    sk = pytest.importorskip("sklearn.neural_network")
+    rng = np.random.default_rng(9)
+    n, d, H = 24, 5, 7
+    X = rng.normal(size=(n, d))
+    y = (np.arange(n) % C).astype(np.float64) if task == 0 else rng.normal(size=n)
+    alpha, lr, mom = 0.21, 0.05, 0.9
+    kw = dict(hidden_layer_sizes=(H,), activation="relu", solver="sgd", alpha=alpha, batch_size=n,
+              learning_rate="constant", learning_rate_init=lr, momentum=mom, nesterovs_momentum=True,
+              shuffle=False, random_state=0)
+    est = sk.MLPClassifier(**kw) if task == 0 else sk.MLPRegressor(**kw)
+    if task == 0:
+        est.partial_fit(X, y.astype(int), classes=np.arange(C))
+    else:
+        est.partial_fit(X, y)
+    opt = getattr(est, "_optimizer", None)
+    if opt is None or not hasattr(opt, "velocities"):
+        pytest.skip("scikit-learn internals differ from the expected layout")
+    P = oracle.param_count(d, H, C)
+    theta0 = rng.normal(0, 0.5, P)
+    W1, c1, W2, c2 = unpack(theta0, d, H, C)
+    est.coefs_[0][...] = W1; est.intercepts_[0][...] = c1
+    est.coefs_[1][...] = W2; est.intercepts_[1][...] = c2
+    for arr in opt.velocities:
+        arr[...] = 0.0
+    steps = 5
+    for _ in range(steps):
+        est.partial_fit(X, y.astype(int)) if task == 0 else est.partial_fit(X, y)
+    theirs = np.concatenate([est.coefs_[0].ravel(), est.intercepts_[0], est.coefs_[1].ravel(), est.intercepts_[1]])
+    th, vel = theta0.copy(), np.zeros(P)
+    for _ in range(steps):
+        g = oracle.loss_grad(1, d, H, C, task, alpha, th, X, y)[1]
+        th, vel = oracle.sgd_steps(1, th, vel, g[None, :], lr, mom)
+    np.testing.assert_allclose(th, theirs, rtol=1e-9, atol=1e-11)
+
+
+def test_sgd_whole_fit_equals_stepwise_replay():
+    # a whole fit with the SGD solver = the minibatch gradients of the checker fed to sgd_steps
+    wl = W.workload("iris8")
+    X, y = wl["X"], wl["y"]
+    cfg = one_config(hidden=6, batch_size=120, epochs=4, alpha=0.01, lr=0.05, beta1=0.7)
+    r = oracle.cv_fits(X, y, 0, 5, cfg, 3, [0], [2], mode=1, want_theta=True, solver=oracle.SOLVER_SGD)
+    _, fo = oracle.fold_split(150, 5, 3)
+    pi = oracle.perm(150, 3, oracle.STREAM_FOLD)
+    train = np.array([row for row in pi if fo[row] != 2])
+    th = oracle.init_params(4, 6, 3, 3, 0, 2).astype(np.float64)
+    vel = np.zeros_like(th)
+    for e in range(4):
+        order = oracle.epoch_order(150, 5, 3, 0, 2, e)
+        assert sorted(order) == sorted(train)
+        g = oracle.loss_grad(1, 4, 6, 3, 0, float(np.float32(0.01)), th, X[order].astype(np.float64), y[order].astype(np.float64))[1]
+        th, vel = oracle.sgd_steps(1, th, vel, g[None, :], np.float32(0.05), np.float32(0.7))
+    np.testing.assert_allclose(r["theta"], th, rtol=1e-12, atol=1e-14)
+
+
+def test_nll_and_mae_scores_recomputed_by_brute_force():
+    sp = pytest.importorskip("scipy.special")
+    wl = W.workload("iris8")
+    X, y = wl["X"], wl["y"]
+    cfg = wl["configs"].copy(); cfg["epochs"] = 7
+    _, fo = oracle.fold_split(150, 5, 0)
+    for mode, tol in ((1, 1e-12), (0, 1e-5)):
+        r = oracle.cv_fits(X, y, 0, 5, cfg, 0, [3], [4], mode=mode, want_theta=True, metric=oracle.METRIC_ALT)
+        W1, b1, W2, b2 = unpack(r["theta"], 4, int(cfg["hidden"][3]), 3)
+        V = np.nonzero(fo == 4)[0]
+        z = np.maximum(X[V].astype(np.float64) @ W1 + b1, 0) @ W2 + b2
+        nll = np.mean(sp.logsumexp(z, axis=1) - z[np.arange(len(V)), y[V].astype(int)])
+        assert abs(r["scores"][0] + nll) < tol * max(1.0, nll)
+        # same training, other metric: identical parameters
+        r2 = oracle.cv_fits(X, y, 0, 5, cfg, 0, [3], [4], mode=mode, want_theta=True)
+        assert np.array_equal(r["theta"], r2["theta"])
+    wl = W.workload("diabetes4096", n_configs=4)
+    X, y = wl["X"], wl["y"]
+    cfg = wl["configs"].copy(); cfg["epochs"] = 5
+    _, fo = oracle.fold_split(442, 5, 0)
+    r = oracle.cv_fits(X, y, 1, 5, cfg, 0, [2], [1], mode=1, want_theta=True, metric=oracle.METRIC_ALT)
+    W1, b1, W2, b2 = unpack(r["theta"], 10, int(cfg["hidden"][2]), 1)
+    V = np.nonzero(fo == 1)[0]
+    z = np.maximum(X[V].astype(np.float64) @ W1 + b1, 0) @ W2 + b2
+    assert abs(r["scores"][0] + np.mean(np.abs(z[:, 0] - y[V]))) < 1e-12
+
+
+def test_nll_at_zero_output_weights_is_log_classes():
+    # a network whose weight matrices are zero predicts (almost) the uniform distribution, so its
+    # NLL is ln C; reached through an L2 strength so large that both matrices collapse to ~0
+    # while the unpenalised biases stay near their small initial values
+    wl = W.workload("iris8")
+    cfg = one_config(hidden=8, batch_size=30, epochs=60, alpha=1e4, lr=1e-3)
+    r = oracle.cv_eval(wl["X"], wl["y"], 0, 5, cfg, 0, mode=1, metric=oracle.METRIC_ALT)
+    assert abs(-r["scores"][0] - np.log(3)) < 0.05
