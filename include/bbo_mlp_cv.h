@@ -46,6 +46,19 @@ typedef struct {
 
 typedef enum { BBO_TASK_CLASSIFICATION = 0, BBO_TASK_REGRESSION = 1 } bbo_task;
 
+/* Update rule of every fit of a handle (paper, Table 1 lists MLP-adam and MLP-sgd).
+ * BBO_SOLVER_SGD is stochastic gradient descent with Nesterov momentum and a constant
+ * learning rate: velocity = momentum*velocity - lr*g; theta += momentum*velocity - lr*g (the
+ * second expression with the new velocity; lr*g rounded once, each expression one fused
+ * multiply-add).  The momentum is the configuration's beta1; beta2 and eps are ignored.     */
+typedef enum { BBO_SOLVER_ADAM = 0, BBO_SOLVER_SGD = 1 } bbo_solver;
+
+/* Held-out score (paper, Table 1: metrics acc, nll for classifiers; mse, mae for regressors).
+ * BBO_METRIC_DEFAULT: accuracy, or minus the mean squared error.  BBO_METRIC_ALT: minus the
+ * mean negative log-likelihood of the true class under the softmax, or minus the mean absolute
+ * error (row sums in ascending row order; NaN maps to -inf).  Always "higher is better".    */
+typedef enum { BBO_METRIC_DEFAULT = 0, BBO_METRIC_ALT = 1 } bbo_metric;
+
 typedef enum {
   BBO_OK = 0,
   BBO_ERR_INVALID_ARG = -1, /* NULL pointer, bad size, hyperparameter or label out of range */
@@ -70,7 +83,8 @@ typedef struct {
                           its random streams: a caller that splits one params_list over several
                           handles (e.g. one per GPU) passes the position of its first entry and
                           gets the scores the unsplit call would give                          */
-  int32_t reserved[2];
+  int32_t solver;      /* a bbo_solver; 0 = Adam                                             */
+  int32_t metric;      /* a bbo_metric; 0 = accuracy / minus mean squared error               */
 } bbo_mlp_cv_options;
 
 /* Creates a handle bound to one device and one stream.  `opt` may be NULL (defaults).

@@ -26,6 +26,8 @@ BBO_ERR_TOO_LARGE = -6
 
 TASK_CLASSIFICATION = 0
 TASK_REGRESSION = 1
+SOLVER_ADAM, SOLVER_SGD = 0, 1
+METRIC_DEFAULT, METRIC_ALT = 0, 1
 
 EXPORTS = [
     "bbo_mlp_cv_create", "bbo_mlp_cv_eval", "bbo_mlp_cv_eval_host", "bbo_mlp_cv_destroy",
@@ -39,7 +41,7 @@ EXPORTS = [
 class Options(ctypes.Structure):
     _fields_ = [("device", ctypes.c_int32), ("stream", ctypes.c_void_p), ("n_classes", ctypes.c_int32),
                 ("trace_steps", ctypes.c_int32), ("keep_theta", ctypes.c_int32),
-                ("config_index_base", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
+                ("config_index_base", ctypes.c_int32), ("solver", ctypes.c_int32), ("metric", ctypes.c_int32)]
 
 
 _lib = None
@@ -102,9 +104,11 @@ def _np_ptr(a):
 
 
 # ---- functions with the C names -------------------------------------------------------
-def bbo_mlp_cv_create(device=-1, stream=0, n_classes=0, trace_steps=0, keep_theta=0, config_index_base=0):
+def bbo_mlp_cv_create(device=-1, stream=0, n_classes=0, trace_steps=0, keep_theta=0, config_index_base=0,
+                      solver=SOLVER_ADAM, metric=METRIC_DEFAULT):
     opt = Options(device=device, stream=stream or None, n_classes=n_classes, trace_steps=trace_steps,
-                  keep_theta=int(keep_theta), config_index_base=int(config_index_base))
+                  keep_theta=int(keep_theta), config_index_base=int(config_index_base), solver=int(solver),
+                  metric=int(metric))
     h = ctypes.c_void_p()
     rc = load().bbo_mlp_cv_create(ctypes.byref(opt), ctypes.byref(h))
     if rc != BBO_OK:
@@ -143,7 +147,8 @@ def bbo_mlp_cv_eval_static(stream_ptr, X_ptr, y_ptr, n, d, task, n_folds, n_clas
 class MlpCv:
     """One handle = one device, one stream, one call in flight."""
 
-    def __init__(self, device=None, stream=None, n_classes=0, trace_steps=0, keep_theta=False, config_index_base=0):
+    def __init__(self, device=None, stream=None, n_classes=0, trace_steps=0, keep_theta=False, config_index_base=0,
+                 solver=SOLVER_ADAM, metric=METRIC_DEFAULT):
         import torch
 
         if not torch.cuda.is_available():
@@ -155,7 +160,8 @@ class MlpCv:
             torch.zeros(1, device="cuda")  # make sure the primary context exists
         self.stream = stream
         sptr = 0 if stream is None else int(stream.cuda_stream)
-        self._h = bbo_mlp_cv_create(self.device, sptr, n_classes, trace_steps, keep_theta, config_index_base)
+        self._h = bbo_mlp_cv_create(self.device, sptr, n_classes, trace_steps, keep_theta, config_index_base,
+                                    solver, metric)
         self._n_configs = self._n_folds = 0
         self.trace_steps = trace_steps
 

@@ -200,7 +200,8 @@ struct FitBuffers {  // device scratch of one evaluation
 // the side streams when there are any.
 int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk, const float* y, int n, int d,
                     int C, int K, int task, const bbo_mlp_config* configs, int n_configs, uint64_t seed,
-                    int trace_steps, int maxB, int config_base, int* launches, cudaError_t* cuda_err) {
+                    int trace_steps, int maxB, int config_base, int solver, int metric, int* launches,
+                    cudaError_t* cuda_err) {
   *cuda_err = cudaSuccess;
   const int n_fits = n_configs * K;
   struct Item { int tier; int Hs; double cost; int id; };
@@ -262,6 +263,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     a.X = Xk; a.y = y; a.pi = buf.pi; a.configs = buf.configs; a.fits = buf.fits + g.begin;
     a.fold_scores = buf.fold_scores; a.trace = buf.trace; a.keep_theta = buf.keep_theta;
     a.n_fits = g.count; a.n_configs = n_configs; a.config_base = config_base;
+    a.solver = solver; a.metric = metric;
     a.n = n; a.d = d; a.dp = g.plan.dp; a.C = C; a.CS = g.plan.CS; a.K = K; a.task = task;
     a.Hs = g.plan.Hs; a.TB = g.plan.TB; a.trace_steps = trace_steps; a.loss_cap = g.plan.loss_cap;
     a.order_bytes = g.plan.order_bytes; a.seed = seed;
@@ -321,7 +323,8 @@ int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out) {
   }
   int dev = o.device;
   if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return BBO_ERR_CUDA;
-  if (dev >= count || o.n_classes < 0 || o.n_classes > kMaxClasses || o.trace_steps < 0 || o.config_index_base < 0)
+  if (dev >= count || o.n_classes < 0 || o.n_classes > kMaxClasses || o.trace_steps < 0 || o.config_index_base < 0 ||
+      o.solver < 0 || o.solver > BBO_SOLVER_SGD || o.metric < 0 || o.metric > BBO_METRIC_ALT)
     return BBO_ERR_INVALID_ARG;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return BBO_ERR_CUDA;
@@ -454,7 +457,7 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   BBO_CUDA(h, cudaEventRecord(h->evf0, s));
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, h->opt.trace_steps, maxB,
-                       h->opt.config_index_base, &launches, &cuda_err);
+                       h->opt.config_index_base, h->opt.solver, h->opt.metric, &launches, &cuda_err);
   if (rc == BBO_ERR_CUDA) return cuda_fail(h, cuda_err, "launch_all_fits");
   if (rc != BBO_OK) return rc;
   BBO_CUDA(h, cudaEventRecord(h->evf1, s));
@@ -760,7 +763,8 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
   FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr};
   int launches = 0;
   cudaError_t cuda_err = cudaSuccess;
-  rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, 0, &launches, &cuda_err);
+  rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, 0, BBO_SOLVER_ADAM,
+                       BBO_METRIC_DEFAULT, &launches, &cuda_err);
   if (rc != BBO_OK) return rc;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(fold_scores, n_configs, K, out_scores);
   if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return BBO_ERR_CUDA;

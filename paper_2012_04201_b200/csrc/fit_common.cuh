@@ -28,6 +28,8 @@ struct FitArgs {
   int32_t n, d, dp, C, CS, K, task;
   int32_t Hs;            // padded hidden width shared by every fit of this launch
   int32_t TB;            // rows per sub-tile (multiple of 4, at most 32)
+  int32_t solver;        // 0 Adam, 1 SGD with Nesterov momentum (momentum = beta1)
+  int32_t metric;        // 0 accuracy / -MSE, 1 -NLL / -MAE
   int32_t trace_steps, loss_cap;  // loss_cap: rows of the per-row loss buffer
   int32_t order_bytes;   // bytes reserved for the epoch order (uint16 per training row)
   uint64_t seed;

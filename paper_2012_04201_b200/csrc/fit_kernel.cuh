@@ -233,6 +233,20 @@ __device__ __forceinline__ void adam_params_ieee(float (&th)[N], const float (&m
   }
 }
 
+// Momentum SGD with Nesterov look-ahead on N parameters held in registers (vel: the velocity,
+// kept where Adam keeps its first moments): vel = momentum vel - lr g;
+// theta += momentum vel - lr g with the new velocity; lr g rounded once.
+template <int N>
+__device__ __forceinline__ void sgd_group(float (&th)[N], float (&vel)[N], const float (&g)[N], float lr,
+                                          float momentum) {
+#pragma unroll
+  for (int e = 0; e < N; ++e) {
+    const float t = __fmul_rn(lr, g[e]);
+    vel[e] = __fmaf_rn(momentum, vel[e], -t);
+    th[e] = __fadd_rn(th[e], __fmaf_rn(momentum, vel[e], -t));
+  }
+}
+
 // Operands of one row of the W1 gradient tile: x[b][k0..k0+7] and delta1[b][jA..jA+3, jB..jB+3].
 struct GradOperands {
   float4 x0, x1, dA, dB;
@@ -262,10 +276,45 @@ struct BlockShared {  // block-wide scalars
 #endif
 };
 
+// Softmax statistics of one row from the logits held by a lane pair: the running maximum and
+// the denominator are taken over the classes in ascending order; the odd lane continues both
+// scans from the even lane's result, and both lanes end up with the row's values.  All 32 lanes
+// must call it.
+template <int CT>
+__device__ __forceinline__ void softmax_scan(const OutLane<CT>& ol, const float (&z)[OutLane<CT>::QA], float& mx,
+                                             float (&ex)[OutLane<CT>::QA], float& sum) {
+  constexpr int QA = OutLane<CT>::QA;
+  const int lane = threadIdx.x & 31;
+  // maximum: ascending scan with strict >, started by the even lane
+  mx = z[0];
+#pragma unroll
+  for (int q = 1; q < QA; ++q) if (z[q] > mx) mx = z[q];
+  const float m_even = __shfl_sync(0xffffffffu, mx, lane & ~1);
+  if (ol.half) {
+    mx = m_even;
+#pragma unroll
+    for (int q = 0; q < QA; ++q) if (q < ol.nq && z[q] > mx) mx = z[q];
+  }
+  mx = __shfl_sync(0xffffffffu, mx, lane | 1);
+#pragma unroll
+  for (int q = 0; q < QA; ++q) ex[q] = spec_expf(__fsub_rn(z[q], mx));
+  // denominator: ascending sum from zero, continued by the odd lane
+  sum = 0.f;
+  if (!ol.half) {
+#pragma unroll
+    for (int q = 0; q < QA; ++q) sum = __fadd_rn(sum, ex[q]);
+  }
+  const float s_even = __shfl_sync(0xffffffffu, sum, lane & ~1);
+  if (ol.half) {
+    sum = s_even;
+#pragma unroll
+    for (int q = 0; q < QA; ++q) if (q < ol.nq) sum = __fadd_rn(sum, ex[q]);
+  }
+  sum = __shfl_sync(0xffffffffu, sum, lane | 1);
+}
+
 // Loss derivative of one row from the logits held by a lane pair, written to D2[row][:].
-// Classification: running maximum and softmax denominator are taken over the classes in
-// ascending order; the odd lane continues both scans from the even lane's result.  All 32 lanes
-// must call it; `active` gates the stores.
+// All 32 lanes must call it; `active` gates the stores.
 template <int CT>
 __device__ __forceinline__ void row_delta(const FitView& v, int task, int CS, const OutLane<CT>& ol,
                                           const float (&z)[OutLane<CT>::QA], float yv, int row, bool active, float invB,
@@ -273,33 +322,8 @@ __device__ __forceinline__ void row_delta(const FitView& v, int task, int CS, co
   constexpr int QA = OutLane<CT>::QA;
   if (task == 0) {
     const int label = (int)yv;
-    // maximum: ascending scan with strict >, started by the even lane
-    float mx = z[0];
-#pragma unroll
-    for (int q = 1; q < QA; ++q) if (z[q] > mx) mx = z[q];
-    const float m_even = __shfl_sync(0xffffffffu, mx, (threadIdx.x & 31) & ~1);
-    if (ol.half) {
-      mx = m_even;
-#pragma unroll
-      for (int q = 0; q < QA; ++q) if (q < ol.nq && z[q] > mx) mx = z[q];
-    }
-    mx = __shfl_sync(0xffffffffu, mx, (threadIdx.x & 31) | 1);
-    float ex[QA];
-#pragma unroll
-    for (int q = 0; q < QA; ++q) ex[q] = spec_expf(__fsub_rn(z[q], mx));
-    // denominator: ascending sum from zero, continued by the odd lane
-    float sum = 0.f;
-    if (!ol.half) {
-#pragma unroll
-      for (int q = 0; q < QA; ++q) sum = __fadd_rn(sum, ex[q]);
-    }
-    const float s_even = __shfl_sync(0xffffffffu, sum, (threadIdx.x & 31) & ~1);
-    if (ol.half) {
-      sum = s_even;
-#pragma unroll
-      for (int q = 0; q < QA; ++q) if (q < ol.nq) sum = __fadd_rn(sum, ex[q]);
-    }
-    sum = __shfl_sync(0xffffffffu, sum, (threadIdx.x & 31) | 1);
+    float mx, sum, ex[QA];
+    softmax_scan<CT>(ol, z, mx, ex, sum);
     // probabilities: branch-free division first; the IEEE routine only where it cannot be certified
     float pr[QA];
     uint32_t safe = 1u;
@@ -581,7 +605,28 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 
       // ---- L2 term and Adam, by the owner of each gradient ----
       const float step = sh.step[step_no & 1];
-      if (has_tile) {
+      const bool sgd = a.solver == 1;
+      if (has_tile && sgd) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int k = k0 + i;
+          if (k < d) {
+            const int offA = L.oW1 + k * Hs + jA, offB = L.oW1 + k * Hs + jB;
+            const float4 wA = *reinterpret_cast<float4*>(v.W + offA), wB = *reinterpret_cast<float4*>(v.W + offB);
+            const float4 mA = *reinterpret_cast<float4*>(v.M + offA), mB = *reinterpret_cast<float4*>(v.M + offB);
+            float w8[8] = {wA.x, wA.y, wA.z, wA.w, wB.x, wB.y, wB.z, wB.w};
+            float m8[8] = {mA.x, mA.y, mA.z, mA.w, mB.x, mB.y, mB.z, mB.w};
+            float g8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) g8[j] = __fmaf_rn(aB, w8[j], g1[i][j]);
+            sgd_group<8>(w8, m8, g8, c.lr, beta1);
+            *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
+            *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
+            *reinterpret_cast<float4*>(v.M + offA) = make_float4(m8[0], m8[1], m8[2], m8[3]);
+            *reinterpret_cast<float4*>(v.M + offB) = make_float4(m8[4], m8[5], m8[6], m8[7]);
+          }
+        }
+      } else if (has_tile) {
         uint32_t redo = 0u;  // rows of the tile whose fast update could not be certified
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -655,7 +700,9 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         wu[CT] = v.W[L.ob1 + tid]; mu[CT] = v.M[L.ob1 + tid]; vu[CT] = v.V[L.ob1 + tid]; gu[CT] = gb1;
 #pragma unroll
         for (int o = 0; o <= CT; ++o) wold[o] = wu[o];
-        if (!adam_group_fast<CT + 1>(wu, mu, vu, gu, beta1, beta2, omb1, omb2, step, eps, eps_safe)) {
+        if (sgd) {
+          sgd_group<CT + 1>(wu, mu, gu, c.lr, beta1);
+        } else if (!adam_group_fast<CT + 1>(wu, mu, vu, gu, beta1, beta2, omb1, omb2, step, eps, eps_safe)) {
 #pragma unroll
           for (int o = 0; o <= CT; ++o) wu[o] = wold[o];
           adam_params_ieee<CT + 1>(wu, mu, vu, step, eps);
@@ -669,7 +716,14 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       }
       if (o_role) {
         const int off = L.ob2 + oo;
-        adam_one(v.W[off], v.M[off], v.V[off], gb2, beta1, beta2, omb1, omb2, step, eps);
+        if (sgd) {
+          float w1[1] = {v.W[off]}, m1[1] = {v.M[off]};
+          const float g1b[1] = {gb2};
+          sgd_group<1>(w1, m1, g1b, c.lr, beta1);
+          v.W[off] = w1[0]; v.M[off] = m1[0];
+        } else {
+          adam_one(v.W[off], v.M[off], v.V[off], gb2, beta1, beta2, omb1, omb2, step, eps);
+        }
       }
       ++step_no;
       BBO_PHASE(8);
@@ -694,7 +748,15 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       const bool act = brow < nb;
       float z[QA];
       output_logits<CT>(v, L, H, ol, act ? brow : nb - 1, z);
-      if (a.task == 0) {
+      if (a.task == 0 && a.metric == 1) {
+        // negative log-likelihood of the true class, written by the lane that holds its logit
+        float mx, sum, ex[QA];
+        softmax_scan<CT>(ol, z, mx, ex, sum);
+        const int label = act ? (int)v.ys[brow] : -1;
+#pragma unroll
+        for (int q = 0; q < QA; ++q)
+          if (q < ol.nq && ol.o0 + q == label) v.D2[brow * CS] = __fsub_rn(logf(sum), __fsub_rn(z[q], mx));
+      } else if (a.task == 0) {
         // prediction: ascending scan with strict >, started by the even lane, finished by the odd one
         float best = z[0];
         int besti = ol.o0;
@@ -714,16 +776,17 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       }
     }
     __syncthreads();
-    if (a.task != 0 && tid == 0) {
+    if ((a.task != 0 || a.metric == 1) && tid == 0) {  // row sums in ascending row order
       float sq = sh.sq;
-      for (int b = 0; b < nb; ++b) { const float r = v.D2[b * CS]; sq = __fmaf_rn(r, r, sq); }
+      if (a.metric == 1) for (int b = 0; b < nb; ++b) sq = __fadd_rn(sq, fabsf(v.D2[b * CS]));
+      else for (int b = 0; b < nb; ++b) { const float r = v.D2[b * CS]; sq = __fmaf_rn(r, r, sq); }
       sh.sq = sq;
     }
     __syncthreads();
   }
   if (tid == 0) {
     float score;
-    if (a.task == 0) {
+    if (a.task == 0 && a.metric == 0) {
       score = __fdiv_rn((float)sh.correct, (float)vs);
     } else {
       score = -__fdiv_rn(sh.sq, (float)vs);
