@@ -50,13 +50,15 @@ def parse_args():
     ap.add_argument("--hidden", type=int, default=0, help="fixed hidden width (0 = U{50..200})")
     ap.add_argument("--batch", type=int, default=0, help="fixed batch size (0 = U{10..250})")
     ap.add_argument("--epochs", type=int, default=200)
+    ap.add_argument("--workload", default="digits_sweep", choices=["digits_sweep", "housing10k", "collider10k"],
+                    help="digits_sweep is the headline cell; the 10,000-row shapes are extra cells")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
 
 def make_workload(args, rank):
     n_configs = max(1, args.fits // 5)
-    wl = workloads.workload("digits_sweep", seed=rank, n_configs=n_configs,
+    wl = workloads.workload(args.workload, seed=rank, n_configs=n_configs,
                             hidden=args.hidden or None, batch_size=args.batch or None, epochs=args.epochs)
     return wl
 
@@ -211,7 +213,8 @@ def run_reference(args, rank, world):
 
 
 def workload_config(args, wl, work):
-    return {"workload": "digits_sweep", "n": int(wl["X"].shape[0]), "d": int(wl["X"].shape[1]), "classes": 10,
+    return {"workload": args.workload, "n": int(wl["X"].shape[0]), "d": int(wl["X"].shape[1]),
+            "classes": 1 if wl["task"] == 1 else int(wl["y"].max()) + 1,
             "n_folds": 5, "epochs": int(args.epochs), "fits_per_step": int(work["n_fits"]),
             "hidden": args.hidden or "U{50..200}", "batch_size": args.batch or "U{10..250}",
             "l2_between_steps": "flushed (256 MiB write)", "variant": "fp32-cuda-core, one CTA per fit, one launch per hidden-width group"}

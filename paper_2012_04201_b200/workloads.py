@@ -135,6 +135,35 @@ def linear_diabetes_shaped(seed=0):
     return X.astype(np.float32), y.astype(np.float32)
 
 
+def housing_shaped(seed=0):
+    """10,000 x 8 regression (the shape of the paper's down-sampled 10,000-row sets): standardised
+    features, half of them log-normal before standardisation (skewed, as counts and incomes
+    are), target = a smooth non-linear function of three features plus N(0, 0.3^2),
+    standardised."""
+    rng = np.random.default_rng(seed)
+    n, d = 10000, 8
+    X = rng.normal(size=(n, d))
+    X[:, :4] = np.exp(0.5 * X[:, :4])
+    X = (X - X.mean(0)) / X.std(0)
+    w = rng.normal(size=d)
+    y = X @ w * 0.5 + np.tanh(X[:, 0] * X[:, 5]) + 0.5 * np.abs(X[:, 6]) + rng.normal(0.0, 0.3, size=n)
+    y = (y - y.mean()) / y.std()
+    return X.astype(np.float32), y.astype(np.float32)
+
+
+def collider_shaped(seed=0):
+    """10,000 x 28, two classes (about 47 / 53): standardised features whose class difference is
+    a weak shift in a few coordinates plus a product term, so that a linear model gets about
+    two thirds right (a hard, noisy binary problem of that shape)."""
+    rng = np.random.default_rng(seed)
+    n, d = 10000, 28
+    X = rng.normal(size=(n, d))
+    score = 0.6 * X[:, 0] - 0.5 * X[:, 3] + 0.7 * X[:, 1] * X[:, 2] + 0.4 * np.abs(X[:, 7]) + rng.normal(0.0, 1.0, size=n)
+    y = (score > np.quantile(score, 0.47)).astype(np.float64)
+    X = (X - X.mean(0)) / X.std(0)
+    return X.astype(np.float32), y.astype(np.float32)
+
+
 def workload(name, seed=0, n_configs=None, hidden=None, batch_size=None, epochs=None):
     """Named workloads.  Returns a dict with X, y, task, n_folds, configs, seed.
 
@@ -144,6 +173,8 @@ def workload(name, seed=0, n_configs=None, hidden=None, batch_size=None, epochs=
     ``diabetes4096`` 442x10 regression, 4096 configs (32 x 128), 200 epochs
     ``digits_sweep`` the digits shape with caller-chosen n_configs / hidden /
     batch_size (throughput sweep)
+    ``housing10k`` 10000x8 regression, ``collider10k`` 10000x28x2: the 10,000-row shape of the
+    paper's down-sampled sets, 128 configs, 50 epochs
     """
     table = {
         "iris8": (blobs_iris_shaped, TASK_CLASSIFICATION, 8, 100, 150),
@@ -151,6 +182,8 @@ def workload(name, seed=0, n_configs=None, hidden=None, batch_size=None, epochs=
         "digits2048": (digits_shaped, TASK_CLASSIFICATION, 2048, 200, 250),
         "diabetes4096": (linear_diabetes_shaped, TASK_REGRESSION, 4096, 200, 250),
         "digits_sweep": (digits_shaped, TASK_CLASSIFICATION, 3200, 200, 250),
+        "housing10k": (housing_shaped, TASK_REGRESSION, 128, 50, 250),
+        "collider10k": (collider_shaped, TASK_CLASSIFICATION, 128, 50, 250),
     }
     gen, task, n_def, e_def, b_hi = table[name]
     X, y = gen(seed)

@@ -89,6 +89,27 @@ def test_nll_and_mae_metrics_match_checker(binding, name, n_cfg, epochs, solver)
         assert not np.array_equal(gpu["fold_scores"], base["fold_scores"])
 
 
+@pytest.mark.parametrize("name", ["housing10k", "collider10k"])
+def test_ten_thousand_row_shape_matches_checker(binding, name):
+    # the shape of the paper's down-sampled 10,000-row sets: 8,000-row training folds, so the
+    # per-epoch permutation sorts 8,000 keys and a fit takes up to 800 steps per epoch
+    wl = W.workload(name, n_configs=12, epochs=3)
+    cfg = wl["configs"]
+    h = binding.MlpCv()
+    for config, fold, epoch in [(0, 0, 0), (11, 4, 2)]:
+        fo, order = h.debug_indices(10000, 5, wl["seed"], config, fold, epoch)
+        assert np.array_equal(fo, oracle.fold_split(10000, 5, wl["seed"])[1])
+        assert np.array_equal(order, oracle.epoch_order(10000, 5, wl["seed"], config, fold, epoch))
+    h.close()
+    gpu = gpu_eval(binding, wl, cfg, trace_steps=50, keep_theta=True)
+    ref = oracle.cv_eval(wl["X"], wl["y"], wl["task"], 5, cfg, wl["seed"], trace_steps=50)
+    exact = check_against_oracle(gpu, ref, name)
+    th = oracle.cv_fits(wl["X"], wl["y"], wl["task"], 5, cfg, wl["seed"], [11], [4], want_theta=True)["theta"]
+    print(f"[{name}] fold scores bit-equal {exact:.3f}; final parameters bit-equal:",
+          np.array_equal(gpu["theta"].astype(np.float64), th))
+    np.testing.assert_allclose(gpu["theta"], th, rtol=1e-3, atol=1e-4)
+
+
 def test_option_values_are_validated(binding):
     with pytest.raises(binding.BboError):
         binding.MlpCv(solver=2)
