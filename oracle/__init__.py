@@ -84,6 +84,11 @@ def lib():
         L.oracle_mlp_cv_eval_ex.restype = ctypes.c_int
         L.oracle_sgd_steps.argtypes = [i32, i64, i32, f64, f64, vp, vp, vp]
         L.oracle_sgd_steps.restype = None
+        L.oracle_mlp_holdout_eval.argtypes = [i32, vp, vp, i64, vp, vp, i64, i32, i32, vp, i32, u64, i32, i32, i32,
+                                              i32, vp, vp]
+        L.oracle_mlp_holdout_eval.restype = ctypes.c_int
+        L.oracle_holdout_order.argtypes = [i64, u64, i32, i32, vp]
+        L.oracle_holdout_order.restype = ctypes.c_int
         L.oracle_num_procs.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -234,6 +239,36 @@ def cv_eval(X, y, task, n_folds, configs, seed, mode=MODE_F32, n_classes=0, trac
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return dict(scores=scores, fold_scores=fold_scores, trace=trace)
+
+
+HOLDOUT_FOLD_KEY = 0xFFFF
+
+
+def holdout_eval(X, y, Xtest, ytest, task, configs, seed, mode=MODE_F32, n_classes=0, n_threads=0,
+                 solver=SOLVER_ADAM, metric=METRIC_DEFAULT, want_theta=False):
+    """One fit per configuration on all rows of (X, y), scored on (Xtest, ytest).
+    Returns dict(scores, theta) (theta: parameters of the last configuration's fit)."""
+    X, y, configs = _prep(X, y, configs)
+    Xtest = np.ascontiguousarray(Xtest, np.float32)
+    ytest = np.ascontiguousarray(ytest, np.float32)
+    n, d = X.shape
+    scores = np.zeros(configs.size, np.float64)
+    theta = None
+    if want_theta:
+        C = 1 if task == 1 else (n_classes or int(max(y.max(), ytest.max())) + 1)
+        theta = np.zeros(param_count(d, int(configs["hidden"][-1]), C), np.float64)
+    rc = lib().oracle_mlp_holdout_eval(mode, _p(X), _p(y), n, _p(Xtest), _p(ytest), Xtest.shape[0], d, task,
+                                       _p(configs), configs.size, seed, n_classes, solver, metric, n_threads,
+                                       _p(scores), _p(theta))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return dict(scores=scores, theta=theta)
+
+
+def holdout_order(n, seed, config, epoch):
+    out = np.zeros(n, np.int32)
+    assert lib().oracle_holdout_order(n, seed, config, epoch, _p(out)) == 0
+    return out
 
 
 def num_procs():

@@ -339,12 +339,17 @@ template <typename T>
 double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, int32_t task,
                int32_t K, const Config& cf, uint32_t config, uint32_t fold, uint64_t seed,
                const std::vector<int32_t>& pi, int32_t trace_steps, double* trace, double* theta_out,
-               int32_t solver = SOLVER_ADAM, int32_t metric = METRIC_DEFAULT) {
-  int64_t vb, vs;
-  fold_segment(n, K, (int32_t)fold, &vb, &vs);
+               int32_t solver = SOLVER_ADAM, int32_t metric = METRIC_DEFAULT, const float* Xtest = nullptr,
+               const float* ytest = nullptr, int64_t n_test = 0) {
+  // Hold-out mode (Xtest given; paper sec. 6.2: the generalisation score is taken on data held
+  // out from the optimisation): train on every row, in the order of the fold permutation, and
+  // score the rows of (Xtest, ytest) in their own order.  `fold` then only keys the random streams.
+  int64_t vb = 0, vs = 0;
+  if (!Xtest) fold_segment(n, K, (int32_t)fold, &vb, &vs);
   std::vector<int32_t> val(pi.begin() + vb, pi.begin() + vb + vs), train;
   train.reserve((size_t)(n - vs));
   for (int64_t i = 0; i < n; ++i) if (i < vb || i >= vb + vs) train.push_back(pi[i]);
+  if (Xtest) { val.resize((size_t)n_test); for (int64_t i = 0; i < n_test; ++i) val[(size_t)i] = (int32_t)i; }
   const int32_t n_tr = (int32_t)train.size();
   const int32_t B = std::min(cf.batch_size, n_tr);
   Shape s{d, cf.hidden, C};
@@ -375,7 +380,8 @@ double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, 
     }
   }
   if (theta_out) for (int64_t i = 0; i < P; ++i) theta_out[i] = (double)th[i];
-  return (double)score_rows<T>(s, task, metric, th.data(), X, y, val.data(), (int32_t)val.size());
+  return (double)score_rows<T>(s, task, metric, th.data(), Xtest ? Xtest : X, Xtest ? ytest : y, val.data(),
+                               (int32_t)val.size());
 }
 
 int validate(const float* X, const float* y, int64_t n, int32_t d, int32_t task, int32_t K,
@@ -587,6 +593,50 @@ int oracle_mlp_cv_eval(int32_t mode, const float* X, const float* y, int64_t n, 
                        double* fold_scores, double* loss_trace) {
   return oracle_mlp_cv_eval_ex(mode, X, y, n, d, task, n_folds, configs, n_configs, seed, n_classes, trace_steps,
                                n_threads, out_scores, fold_scores, loss_trace, 0, 0);
+}
+
+// Hold-out evaluation (paper sec. 6.2): one fit per configuration, trained on all n rows and scored
+// on the n_test rows of (Xtest, ytest).  The random streams of these fits use the fold index
+// HOLDOUT_FOLD_KEY, which no cross-validation fold can have.  theta_out: parameters of the last
+// configuration's fit (or null).
+enum : uint32_t { HOLDOUT_FOLD_KEY = 0xFFFFu };
+int oracle_mlp_holdout_eval(int32_t mode, const float* X, const float* y, int64_t n, const float* Xtest,
+                            const float* ytest, int64_t n_test, int32_t d, int32_t task, const void* configs,
+                            int32_t n_configs, uint64_t seed, int32_t n_classes, int32_t solver, int32_t metric,
+                            int32_t n_threads, double* out_scores, double* theta_out) {
+  const Config* cfg = (const Config*)configs;
+  if (!Xtest || !ytest || n_test < 1 || validate(X, y, n, d, task, 2, cfg, n_configs) != 0) return -1;
+  if (solver < 0 || solver > 1 || metric < 0 || metric > 1) return -1;
+  int32_t C = derive_classes(y, n, task, n_classes);
+  if (C < 1) return -1;
+  if (task == 0 && n_classes == 0) {  // labels of the test rows may exceed those seen in training
+    const int32_t Ct = derive_classes(ytest, n_test, task, 0);
+    if (Ct < 1) return -1;
+    if (Ct > C) C = Ct;
+  }
+  std::vector<int32_t> pi;
+  rng_perm((int32_t)n, seed, STREAM_FOLD, 0, 0, 0, pi);
+#ifdef _OPENMP
+  if (n_threads <= 0) n_threads = omp_get_num_procs();
+#pragma omp parallel for schedule(dynamic, 1) num_threads(n_threads)
+#endif
+  for (int32_t c = 0; c < n_configs; ++c) {
+    double* tho = (theta_out && c == n_configs - 1) ? theta_out : nullptr;
+    out_scores[c] = mode == 1
+        ? run_fit<double>(X, y, n, d, C, task, 1, cfg[c], c, HOLDOUT_FOLD_KEY, seed, pi, 0, nullptr, tho, solver, metric, Xtest, ytest, n_test)
+        : run_fit<float>(X, y, n, d, C, task, 1, cfg[c], c, HOLDOUT_FOLD_KEY, seed, pi, 0, nullptr, tho, solver, metric, Xtest, ytest, n_test);
+  }
+  return 0;
+}
+
+// Epoch order of a hold-out fit: the epoch permutation applied to the whole fold permutation.
+int oracle_holdout_order(int64_t n, uint64_t seed, int32_t config, int32_t epoch, int32_t* out) {
+  if (n < 1) return -1;
+  std::vector<int32_t> pi, sigma;
+  rng_perm((int32_t)n, seed, STREAM_FOLD, 0, 0, 0, pi);
+  rng_perm((int32_t)n, seed, STREAM_PERM, (uint32_t)config, HOLDOUT_FOLD_KEY, (uint32_t)epoch, sigma);
+  for (int64_t i = 0; i < n; ++i) out[i] = pi[sigma[(size_t)i]];
+  return 0;
 }
 
 // n_steps momentum-SGD updates on P parameters with caller-supplied gradients grads[n_steps][P].

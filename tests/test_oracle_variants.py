@@ -137,3 +137,43 @@ def test_nll_at_zero_output_weights_is_log_classes():
     cfg = one_config(hidden=8, batch_size=30, epochs=60, alpha=1e4, lr=1e-3)
     r = oracle.cv_eval(wl["X"], wl["y"], 0, 5, cfg, 0, mode=1, metric=oracle.METRIC_ALT)
     assert abs(-r["scores"][0] - np.log(3)) < 0.05
+
+
+def test_holdout_fit_trains_on_all_rows_and_scores_the_test_rows():
+    # paper sec. 6.2: the generalisation score comes from rows held out of the optimisation
+    wl = W.workload("iris8")
+    X, y = wl["X"], wl["y"]
+    Xtr, ytr, Xte, yte = X[:110], y[:110], X[110:], y[110:]
+    cfg = one_config(hidden=6, batch_size=110, epochs=4, alpha=0.01, lr=0.05, beta1=0.7, beta2=0.9)
+    r = oracle.holdout_eval(Xtr, ytr, Xte, yte, 0, cfg, 5, mode=1, want_theta=True)
+    # (a) the training is the stepwise replay over all 110 rows in the stated order
+    th = oracle.init_params(4, 6, 3, 5, 0, oracle.HOLDOUT_FOLD_KEY).astype(np.float64)
+    grads = []
+    for e in range(4):
+        order = oracle.holdout_order(110, 5, 0, e)
+        assert sorted(order) == list(range(110))
+        th_e, _, _ = (oracle.adam_steps(1, th, np.zeros_like(th), np.zeros_like(th), np.array(grads),
+                                        float(np.float32(0.05)), float(np.float32(0.7)), float(np.float32(0.9)),
+                                        float(np.float32(1e-8))) if grads else (th, None, None))
+        grads.append(oracle.loss_grad(1, 4, 6, 3, 0, float(np.float32(0.01)), th_e, Xtr[order].astype(np.float64),
+                                      ytr[order].astype(np.float64))[1])
+    th_final, _, _ = oracle.adam_steps(1, th, np.zeros_like(th), np.zeros_like(th), np.array(grads),
+                                       float(np.float32(0.05)), float(np.float32(0.7)), float(np.float32(0.9)),
+                                       float(np.float32(1e-8)))
+    np.testing.assert_allclose(r["theta"], th_final, rtol=1e-12, atol=1e-14)
+    # (b) the score is the accuracy of those parameters on the test rows
+    W1, b1, W2, b2 = unpack(r["theta"], 4, 6, 3)
+    z = np.maximum(Xte.astype(np.float64) @ W1 + b1, 0) @ W2 + b2
+    assert abs(r["scores"][0] - np.mean(np.argmax(z, 1) == yte)) < 1e-12
+    # (c) it does not depend on the test rows' content beyond the score, nor on other configurations
+    cfg2 = np.concatenate([cfg, one_config(hidden=9, epochs=2)])
+    r2 = oracle.holdout_eval(Xtr, ytr, Xte[::-1].copy(), yte[::-1].copy(), 0, cfg2, 5, mode=1)
+    assert abs(r2["scores"][0] - r["scores"][0]) < 1e-12
+    # regression with the mae metric, float mode
+    wl = W.workload("diabetes4096", n_configs=3)
+    X, y = wl["X"], wl["y"]
+    cfg = wl["configs"].copy(); cfg["epochs"] = 4
+    r = oracle.holdout_eval(X[:400], y[:400], X[400:], y[400:], 1, cfg, 0, metric=oracle.METRIC_ALT, want_theta=True)
+    W1, b1, W2, b2 = unpack(r["theta"], 10, int(cfg["hidden"][-1]), 1)
+    z = np.maximum(X[400:].astype(np.float64) @ W1 + b1, 0) @ W2 + b2
+    assert abs(r["scores"][-1] + np.mean(np.abs(z[:, 0] - y[400:]))) < 1e-5
