@@ -108,6 +108,20 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, in
                     int32_t task, int32_t n_folds, const bbo_mlp_config* configs,
                     int32_t n_configs, uint64_t seed, float* out_scores);
 
+/* Hold-out ("generalisation") scores of the same configurations (paper, sec. 6.2: the data
+ * are split into the part the optimizers see through cross-validation and a part held out to
+ * measure generalisation).  One fit per configuration: trained on all n rows of (X, y), in the
+ * order of the fold permutation of `seed`, with the minibatch and initialisation streams keyed
+ * by fold index 65535, then scored on the n_test rows of (Xtest, ytest) in their own order.
+ *   X, y, Xtest, ytest  DEVICE, layouts as in bbo_mlp_cv_eval; n_test in [1, row cap]
+ *   out_scores          DEVICE [n_configs]: the handle's metric on the test rows
+ * The class count covers the labels of both parts.  Ownership, synchrony and errors as in
+ * bbo_mlp_cv_eval; bbo_mlp_cv_fold_scores then returns one value per configuration.        */
+int bbo_mlp_cv_eval_holdout(bbo_mlp_cv* h, const float* X, const float* y, int64_t n,
+                            const float* Xtest, const float* ytest, int64_t n_test, int32_t d,
+                            int32_t task, const bbo_mlp_config* configs, int32_t n_configs,
+                            uint64_t seed, float* out_scores);
+
 /* As bbo_mlp_cv_eval, with X, y and out_scores in HOST memory: copies them to device
  * scratch owned by the handle, evaluates, copies the scores back.                         */
 int bbo_mlp_cv_eval_host(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d,

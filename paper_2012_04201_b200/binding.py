@@ -30,7 +30,7 @@ SOLVER_ADAM, SOLVER_SGD = 0, 1
 METRIC_DEFAULT, METRIC_ALT = 0, 1
 
 EXPORTS = [
-    "bbo_mlp_cv_create", "bbo_mlp_cv_eval", "bbo_mlp_cv_eval_host", "bbo_mlp_cv_destroy",
+    "bbo_mlp_cv_create", "bbo_mlp_cv_eval", "bbo_mlp_cv_eval_host", "bbo_mlp_cv_eval_holdout", "bbo_mlp_cv_destroy",
     "bbo_mlp_cv_fold_scores", "bbo_mlp_cv_loss_trace", "bbo_mlp_cv_debug_theta",
     "bbo_mlp_cv_debug_indices", "bbo_mlp_cv_debug_rng", "bbo_mlp_cv_debug_exp",
     "bbo_mlp_cv_query_caps", "bbo_mlp_cv_last_timing", "bbo_mlp_cv_strerror",
@@ -69,6 +69,7 @@ def load():
     L.bbo_mlp_cv_create.argtypes = [ctypes.POINTER(Options), ctypes.POINTER(vp)]
     L.bbo_mlp_cv_eval.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_eval_host.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, i32, u64, vp]
+    L.bbo_mlp_cv_eval_holdout.argtypes = [vp, vp, vp, i64, vp, vp, i64, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_destroy.argtypes = [vp]
     L.bbo_mlp_cv_eval_static.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_fold_scores.argtypes = [vp, vp, i64]
@@ -184,6 +185,25 @@ class MlpCv:
                              configs, seed, out.data_ptr())
         self._check(rc)
         self._n_configs, self._n_folds = configs.size, n_folds
+        return out
+
+    def eval_holdout(self, X, y, Xtest, ytest, task, configs, seed, out=None):
+        """One fit per configuration on all rows of ``X``, scored on ``Xtest`` (CUDA tensors)."""
+        torch = self._torch
+        for t in (X, y, Xtest, ytest):
+            assert t.is_cuda and t.dtype == torch.float32
+        X, y, Xtest, ytest = X.contiguous(), y.contiguous(), Xtest.contiguous(), ytest.contiguous()
+        assert X.shape[1] == Xtest.shape[1]
+        configs = np.ascontiguousarray(configs, dtype=CONFIG_DTYPE)
+        if out is None:
+            out = torch.empty(configs.size, dtype=torch.float32, device=X.device)
+        if self.stream is not None:
+            self.stream.wait_stream(torch.cuda.current_stream(X.device))
+        rc = load().bbo_mlp_cv_eval_holdout(self._h, X.data_ptr(), y.data_ptr(), X.shape[0], Xtest.data_ptr(),
+                                            ytest.data_ptr(), Xtest.shape[0], X.shape[1], task, _np_ptr(configs),
+                                            configs.size, seed, out.data_ptr())
+        self._check(rc)
+        self._n_configs, self._n_folds = configs.size, 1
         return out
 
     def eval_host(self, X, y, task, n_folds, configs, seed):

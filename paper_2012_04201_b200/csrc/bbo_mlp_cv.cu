@@ -56,7 +56,7 @@ struct bbo_mlp_cv {
   // scratch
   DevBuf<bbo::Config> configs;
   DevBuf<int2> fits;
-  DevBuf<float> fold_scores, trace, theta, xpad, hx, hy, hscores, dbg_f;
+  DevBuf<float> fold_scores, trace, theta, xpad, xpad_t, hx, hy, hscores, dbg_f;
   DevBuf<int32_t> pi, misc, dbg_i;
   DevBuf<uint32_t> dbg_u;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr, evf0 = nullptr, evf1 = nullptr;
@@ -136,7 +136,7 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
   p.CS = bbo::round_up(C, 4);
   p.dp = bbo::round_up(d, 8);
   p.Hs = Hs;
-  const int n_tr_max = n - n / K;
+  const int n_tr_max = K == 1 ? n : n - n / K;  // K == 1: hold-out mode, every row trains
   p.order_bytes = bbo::round_up(2 * n_tr_max, 16);
   p.loss_cap = tracing ? std::min(maxB, n_tr_max) : 0;
   p.n_sort = n_tr_max;
@@ -198,10 +198,16 @@ struct FitBuffers {  // device scratch of one evaluation
 // short.  Cost model (SM cycles, from phase timings): per optimizer step 8000 + 80 H fixed
 // (Adam, barriers, chain latencies) plus 2.9 H per row.  One grid per (tier, width) group, on
 // the side streams when there are any.
+struct HoldoutRows {  // hold-out mode: the rows to score (null Xt = cross-validation)
+  const float* Xt = nullptr;
+  const float* yt = nullptr;
+  int n_test = 0;
+};
+
 int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk, const float* y, int n, int d,
                     int C, int K, int task, const bbo_mlp_config* configs, int n_configs, uint64_t seed,
-                    int trace_steps, int maxB, int config_base, int solver, int metric, int* launches,
-                    cudaError_t* cuda_err) {
+                    int trace_steps, int maxB, int config_base, int solver, int metric, const HoldoutRows& ho,
+                    int* launches, cudaError_t* cuda_err) {
   *cuda_err = cudaSuccess;
   const int n_fits = n_configs * K;
   struct Item { int tier; int Hs; double cost; int id; };
@@ -211,6 +217,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     for (int f = 0; f < K; ++f) {
       int vb, vs;
       bbo::fold_segment(n, K, f, &vb, &vs);
+      if (ho.Xt) vs = 0;  // hold-out mode: every row trains
       const double n_tr = n - vs, B = std::min<double>(q.batch_size, n_tr);
       const double steps = (double)q.epochs * std::ceil(n_tr / B);
       const double width = (double)q.hidden * (d + C) / 74.0;  // H for the 64-feature, 10-class shape
@@ -264,6 +271,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     a.fold_scores = buf.fold_scores; a.trace = buf.trace; a.keep_theta = buf.keep_theta;
     a.n_fits = g.count; a.n_configs = n_configs; a.config_base = config_base;
     a.solver = solver; a.metric = metric;
+    a.Xt = ho.Xt; a.yt = ho.yt; a.n_test = ho.n_test;
     a.n = n; a.d = d; a.dp = g.plan.dp; a.C = C; a.CS = g.plan.CS; a.K = K; a.task = task;
     a.Hs = g.plan.Hs; a.TB = g.plan.TB; a.trace_steps = trace_steps; a.loss_cap = g.plan.loss_cap;
     a.order_bytes = g.plan.order_bytes; a.seed = seed;
@@ -359,7 +367,7 @@ int bbo_mlp_cv_destroy(bbo_mlp_cv* h) {
   DeviceGuard g(h->device);
   cudaStreamSynchronize(h->stream);
   h->configs.release(); h->fits.release(); h->fold_scores.release(); h->trace.release();
-  h->theta.release(); h->xpad.release(); h->hx.release(); h->hy.release(); h->hscores.release();
+  h->theta.release(); h->xpad.release(); h->xpad_t.release(); h->hx.release(); h->hy.release(); h->hscores.release();
   h->dbg_f.release(); h->pi.release(); h->misc.release(); h->dbg_i.release(); h->dbg_u.release();
   if (h->ev0) cudaEventDestroy(h->ev0);
   if (h->ev1) cudaEventDestroy(h->ev1);
@@ -374,11 +382,17 @@ int bbo_mlp_cv_destroy(bbo_mlp_cv* h) {
   return BBO_OK;
 }
 
-int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, int32_t d, int32_t task,
-                    int32_t K, const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed,
-                    float* out_scores) {
+// Shared body of the cross-validation and hold-out evaluations.  Xt == null: K-fold
+// cross-validation.  Xt != null: K must be 1; every row of X trains and the n_test rows of
+// (Xt, yt) are scored.
+static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, int32_t d, int32_t task,
+                     int32_t K, const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed,
+                     float* out_scores, const float* Xt, const float* yt, int64_t n_test64) {
   if (!h || !X || !y || !configs || !out_scores) return BBO_ERR_INVALID_ARG;
-  if (n64 < 2 || d < 1 || K < 2 || K > n64 || n_configs < 1) return BBO_ERR_INVALID_ARG;
+  const bool holdout = Xt != nullptr;
+  if (n64 < 2 || d < 1 || n_configs < 1) return BBO_ERR_INVALID_ARG;
+  if (holdout ? (K != 1 || !yt || n_test64 < 1) : (K < 2 || K > n64)) return BBO_ERR_INVALID_ARG;
+  if (holdout && n_test64 > kMaxRows) return BBO_ERR_UNSUPPORTED;
   if (task != BBO_TASK_CLASSIFICATION && task != BBO_TASK_REGRESSION) return BBO_ERR_INVALID_ARG;
   if (n64 > kMaxRows || (int64_t)n_configs * K > (1 << 30) || (int64_t)n_configs + h->opt.config_index_base >= (1 << 28))
     return BBO_ERR_UNSUPPORTED;
@@ -388,7 +402,9 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   DeviceGuard g(h->device);
   if (!is_device_ptr(X, h->device) || !is_device_ptr(y, h->device) || !is_device_ptr(out_scores, h->device))
     return BBO_ERR_INVALID_ARG;
+  if (holdout && (!is_device_ptr(Xt, h->device) || !is_device_ptr(yt, h->device))) return BBO_ERR_INVALID_ARG;
   const int n = (int)n64;
+  const int n_test = holdout ? (int)n_test64 : 0;
   cudaStream_t s = h->stream;
   h->cuda_error.clear();
   h->last_fold_count = h->last_trace_count = h->last_theta_count = 0;
@@ -402,6 +418,11 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
     bbo::label_scan_kernel<<<std::min(64, (n + 255) / 256), 256, 0, s>>>(y, n, h->misc.p + 1);
     BBO_CUDA(h, cudaGetLastError());
     ++launches;
+    if (holdout) {  // the class count covers the labels of the test rows as well
+      bbo::label_scan_kernel<<<std::min(64, (n_test + 255) / 256), 256, 0, s>>>(yt, n_test, h->misc.p + 1);
+      BBO_CUDA(h, cudaGetLastError());
+      ++launches;
+    }
     int32_t info[2];
     BBO_CUDA(h, cudaMemcpyAsync(info, h->misc.p + 1, sizeof(info), cudaMemcpyDeviceToHost, s));
     BBO_CUDA(h, cudaStreamSynchronize(s));
@@ -447,6 +468,18 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
     ++launches;
     Xk = h->xpad.p;
   }
+  HoldoutRows ho;
+  if (holdout) {
+    ho.Xt = Xt; ho.yt = yt; ho.n_test = n_test;
+    if (dp != d || (reinterpret_cast<uintptr_t>(Xt) & 15u) != 0) {
+      const size_t total = (size_t)n_test * dp;
+      BBO_CUDA(h, h->xpad_t.reserve(total));
+      bbo::pad_rows_kernel<<<(int)std::min<size_t>(1024, (total + 255) / 256), 256, 0, s>>>(Xt, n_test, d, dp, h->xpad_t.p);
+      BBO_CUDA(h, cudaGetLastError());
+      ++launches;
+      ho.Xt = h->xpad_t.p;
+    }
+  }
   BBO_CUDA(h, launch_fold_permutation(n, seed, h->pi.p, s));
   ++launches;
 
@@ -457,7 +490,7 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   BBO_CUDA(h, cudaEventRecord(h->evf0, s));
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, h->opt.trace_steps, maxB,
-                       h->opt.config_index_base, h->opt.solver, h->opt.metric, &launches, &cuda_err);
+                       h->opt.config_index_base, h->opt.solver, h->opt.metric, ho, &launches, &cuda_err);
   if (rc == BBO_ERR_CUDA) return cuda_fail(h, cuda_err, "launch_all_fits");
   if (rc != BBO_OK) return rc;
   BBO_CUDA(h, cudaEventRecord(h->evf1, s));
@@ -473,6 +506,18 @@ int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, 
   h->last_trace_count = tracing ? (int64_t)n_fits * h->opt.trace_steps : 0;
   h->last_theta_count = theta_count;
   return BBO_OK;
+}
+
+int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d, int32_t task, int32_t K,
+                    const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed, float* out_scores) {
+  return eval_impl(h, X, y, n, d, task, K, configs, n_configs, seed, out_scores, nullptr, nullptr, 0);
+}
+
+int bbo_mlp_cv_eval_holdout(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, const float* Xtest,
+                            const float* ytest, int64_t n_test, int32_t d, int32_t task,
+                            const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed, float* out_scores) {
+  if (!Xtest || !ytest) return BBO_ERR_INVALID_ARG;
+  return eval_impl(h, X, y, n, d, task, 1, configs, n_configs, seed, out_scores, Xtest, ytest, n_test);
 }
 
 int bbo_mlp_cv_eval_host(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
@@ -764,7 +809,7 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
   int launches = 0;
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, 0, BBO_SOLVER_ADAM,
-                       BBO_METRIC_DEFAULT, &launches, &cuda_err);
+                       BBO_METRIC_DEFAULT, HoldoutRows{}, &launches, &cuda_err);
   if (rc != BBO_OK) return rc;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(fold_scores, n_configs, K, out_scores);
   if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return BBO_ERR_CUDA;

@@ -18,6 +18,9 @@ struct FitArgs {
   const float* X;        // [n][dp], rows 16-byte aligned
   const float* y;        // [n]
   const int32_t* pi;     // [n] fold permutation
+  const float* Xt;       // hold-out mode: test rows [n_test][dp] (null otherwise)
+  const float* yt;       // hold-out mode: test labels / targets [n_test]
+  int32_t n_test;        // hold-out mode: number of test rows (0 otherwise)
   const Config* configs; // [n_configs]
   const int2* fits;      // this launch's (configuration, fold) list, costliest first
   float* fold_scores;    // [n_configs * K]
@@ -60,6 +63,9 @@ __host__ __device__ inline int next_pow2(int x) {
   while (p < x) p <<= 1;
   return p;
 }
+
+// Fold index that keys the random streams of a hold-out fit (no cross-validation fold has it).
+constexpr uint32_t kHoldoutFoldKey = 0xFFFFu;
 
 constexpr int kSortBuckets = 2048;  // power of two
 

@@ -57,17 +57,17 @@ struct FitView {  // per-fit pointers into shared memory
 // Asynchronous gather of nb dataset rows into buffer `buf` of Xs / ys.  Rows nb..TB-1 are
 // zero-filled so that the forward tiles read defined values.  row_of(r) = dataset row.
 template <typename RowFn>
-__device__ __forceinline__ void stage_rows_async(const FitArgs& a, const FitView& v, int dp, int buf, int nb,
-                                                 RowFn row_of, int tid, int nt) {
+__device__ __forceinline__ void stage_rows_async(const FitArgs& a, const float* Xsrc, const float* ysrc, const FitView& v,
+                                                 int dp, int buf, int nb, RowFn row_of, int tid, int nt) {
   const int vec = dp >> 2;
   float* xs = v.Xs + buf * a.TB * dp;
   for (int i = tid; i < a.TB * vec; i += nt) {
     const int r = i / vec, q = i - r * vec;
     float4* dst = reinterpret_cast<float4*>(xs) + i;
-    if (r < nb) cp_async_16(dst, reinterpret_cast<const float4*>(a.X + (size_t)row_of(r) * dp) + q);
+    if (r < nb) cp_async_16(dst, reinterpret_cast<const float4*>(Xsrc + (size_t)row_of(r) * dp) + q);
     else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  for (int r = tid; r < nb; r += nt) cp_async_4(v.ys + buf * a.TB + r, a.y + row_of(r));
+  for (int r = tid; r < nb; r += nt) cp_async_4(v.ys + buf * a.TB + r, ysrc + row_of(r));
   cp_async_commit();
 }
 
@@ -363,9 +363,15 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   const int dp = DPC ? DPC : a.dp;
   const int Hs = HSC ? HSC : a.Hs;
   const Layout L(d, Hs, CT, CS);
-  int vb, vs;
-  fold_segment(a.n, a.K, fold, &vb, &vs);
+  // Hold-out mode (paper sec. 6.2: the generalisation score comes from rows kept out of the
+  // optimisation): every row trains, in the order of the fold permutation, and the score is taken
+  // on the rows of a second matrix; the fold index then only keys the random streams.
+  const bool holdout = a.Xt != nullptr;
+  const uint32_t rng_fold = holdout ? kHoldoutFoldKey : (uint32_t)fold;
+  int vb = 0, vs = 0;
+  if (!holdout) fold_segment(a.n, a.K, fold, &vb, &vs);
   const int n_tr = a.n - vs;
+  if (holdout) vs = a.n_test;  // rows to score
   const int B = c.batch_size < n_tr ? c.batch_size : n_tr;
 
 #ifdef BBO_PHASE_TIMERS
@@ -396,7 +402,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     const float bound2 = __fsqrt_rn(__fdiv_rn(6.0f, (float)(H + CT)));
     const int n1 = d * H, n2 = H * CT;
     for (int blk = tid; blk < ((n1 + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 0u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, rng_fold, 0u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const int idx = 4 * blk + w;
@@ -404,12 +410,12 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       }
     }
     for (int blk = tid; blk < ((H + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 1u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, rng_fold, 1u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) { const int j = 4 * blk + w; if (j < H) v.W[L.ob1 + j] = glorot_value(word_of(r, w), bound1); }
     }
     for (int blk = tid; blk < ((n2 + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 2u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, rng_fold, 2u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const int idx = 4 * blk + w;
@@ -417,7 +423,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       }
     }
     for (int blk = tid; blk < ((CT + 3) >> 2); blk += nt) {
-      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, fold, 3u, blk);
+      const uint4 r = philox4x32_10(a.seed, kStreamInit, rng_config, rng_fold, 3u, blk);
 #pragma unroll
       for (int w = 0; w < 4; ++w) { const int o = 4 * blk + w; if (o < CT) v.W[L.ob2 + o] = glorot_value(word_of(r, w), bound2); }
     }
@@ -449,13 +455,13 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     for (int j = 0; j < 8; ++j) v1[i][j] = 0.f;
 
   for (int e = 0; e < c.epochs; ++e) {
-    build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, vs, a.seed, rng_config, fold, e, tid, nt);
+    build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, holdout ? 0 : vs, a.seed, rng_config, rng_fold, e, tid, nt);
     BBO_PHASE(1);
     int buf = 0;
     {  // first sub-tile of the epoch
       const int Bs0 = n_tr < B ? n_tr : B, nb0 = Bs0 < TB ? Bs0 : TB;
       const uint16_t* rows = v.order;
-      stage_rows_async(a, v, dp, 0, nb0, [&](int r) { return (int)rows[r]; }, tid, nt);
+      stage_rows_async(a, a.X, a.y, v, dp, 0, nb0, [&](int r) { return (int)rows[r]; }, tid, nt);
     }
     for (int s0 = 0; s0 < n_tr; s0 += B) {
       const int Bs = (n_tr - s0) < B ? (n_tr - s0) : B;
@@ -490,7 +496,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           if (ns0 < n_tr) {
             const int nnb = (nBs - nt0) < TB ? (nBs - nt0) : TB;
             const uint16_t* rows = v.order + ns0 + nt0;
-            stage_rows_async(a, v, dp, buf ^ 1, nnb, [&](int r) { return (int)rows[r]; }, tid, nt);
+            stage_rows_async(a, a.X, a.y, v, dp, buf ^ 1, nnb, [&](int r) { return (int)rows[r]; }, tid, nt);
           }
         }
         forward_hidden(v, L, xs, d, dp, Hs, nb, tid, nt);
@@ -738,7 +744,8 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   __syncthreads();
   for (int t0 = 0; t0 < vs; t0 += TB) {
     const int nb = (vs - t0) < TB ? (vs - t0) : TB;
-    stage_rows_async(a, v, dp, 0, nb, [&](int r) { return a.pi[vb + t0 + r]; }, tid, nt);
+    if (holdout) stage_rows_async(a, a.Xt, a.yt, v, dp, 0, nb, [&](int r) { return t0 + r; }, tid, nt);
+    else stage_rows_async(a, a.X, a.y, v, dp, 0, nb, [&](int r) { return a.pi[vb + t0 + r]; }, tid, nt);
     cp_async_wait_all();
     __syncthreads();
     forward_hidden(v, L, v.Xs, d, dp, Hs, nb, tid, nt);

@@ -110,6 +110,34 @@ def test_ten_thousand_row_shape_matches_checker(binding, name):
     np.testing.assert_allclose(gpu["theta"], th, rtol=1e-3, atol=1e-4)
 
 
+@pytest.mark.parametrize("name,n_train,metric,solver", [("iris8", 110, 0, 0), ("digits2048", 1500, 1, 0),
+                                                        ("diabetes4096", 401, 0, 0), ("breast128", 450, 0, 1),
+                                                        ("diabetes4096", 390, 1, 0)])
+def test_holdout_scores_match_checker(binding, name, n_train, metric, solver):
+    # paper sec. 6.2: train on the optimisation part, score the held-out part
+    wl = W.workload(name, n_configs=10) if name != "iris8" else W.workload(name)
+    X, y = wl["X"], wl["y"]
+    cfg = sgd_configs(wl, 8, 6) if solver else wl["configs"][:8].copy()
+    cfg["epochs"] = 6 if name != "digits2048" else 2
+    h = binding.MlpCv(keep_theta=True, solver=solver, metric=metric)
+    Xd, yd = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+    got = h.eval_holdout(Xd[:n_train], yd[:n_train], Xd[n_train:], yd[n_train:], wl["task"], cfg, wl["seed"]).cpu().numpy()
+    C = 1 if wl["task"] == 1 else int(y.max()) + 1
+    theta = h.debug_theta(oracle.param_count(X.shape[1], int(cfg[-1]["hidden"]), C))
+    per_fit = h.fold_scores()
+    h.close()
+    ref = oracle.holdout_eval(X[:n_train], y[:n_train], X[n_train:], y[n_train:], wl["task"], cfg, wl["seed"],
+                              solver=solver, metric=metric, want_theta=True)
+    assert np.array_equal(per_fit.ravel(), got)
+    both_inf = np.isinf(got) & np.isinf(ref["scores"])
+    err = np.where(both_inf, 0.0, np.abs(got.astype(np.float64) - ref["scores"]))
+    print(f"[{name}/holdout] max err {err.max():.3g}, bit-equal {np.mean((got.astype(np.float64) == ref['scores']) | both_inf):.3f};"
+          f" parameters bit-equal: {np.array_equal(theta.astype(np.float64), ref['theta'])}")
+    assert np.mean(err <= 1e-3) >= 0.99
+    fin = np.isfinite(ref["theta"])
+    np.testing.assert_allclose(theta[fin], ref["theta"][fin], rtol=1e-3, atol=1e-4)
+
+
 def test_option_values_are_validated(binding):
     with pytest.raises(binding.BboError):
         binding.MlpCv(solver=2)
