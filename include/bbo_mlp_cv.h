@@ -19,6 +19,10 @@
  * layer, element), so a score depends only on its own configuration, its index in the list
  * and the seed -- never on the other entries, the grid or the scheduling.
  *
+ * Variants selected per handle (bbo_mlp_cv_options): the MLP-sgd update rule and the nll / mae
+ * metrics of the paper's Table 1; bbo_mlp_cv_eval_holdout gives the generalisation score of
+ * sec. 6.2 (train on all rows, score a held-out matrix).
+ *
  * No C++ types, no exceptions and no printing cross this boundary.  Every function returns
  * 0 on success or a negative bbo_status.  All floating point is IEEE binary32 unless noted.
  */
