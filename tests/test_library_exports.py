@@ -29,6 +29,7 @@ def test_strerror_and_argument_checks_without_a_device():
     assert lib.bbo_mlp_cv_create(None, None) == binding.BBO_ERR_INVALID_ARG
     assert lib.bbo_mlp_cv_destroy(None) == binding.BBO_ERR_INVALID_ARG
     assert lib.bbo_mlp_cv_eval(None, None, None, 0, 0, 0, 0, None, 0, 0, None) == binding.BBO_ERR_INVALID_ARG
+    assert lib.bbo_mlp_cv_eval_holdout(None, None, None, 0, None, None, 0, 0, 0, None, 0, 0, None) == binding.BBO_ERR_INVALID_ARG
 
 
 def test_config_layout_matches_header():
