@@ -31,6 +31,7 @@ struct FitArgs {
   int32_t n, d, dp, C, CS, K, task;
   int32_t Hs;            // padded hidden width shared by every fit of this launch
   int32_t TB;            // rows per sub-tile (multiple of 4, at most 32)
+  int32_t extra_warps;   // pipelined schedule: warps after the tile / unit owners that run the output layer
   int32_t solver;        // 0 Adam, 1 SGD with Nesterov momentum (momentum = beta1)
   int32_t metric;        // 0 accuracy / -MSE, 1 -NLL / -MAE
   int32_t trace_steps, loss_cap;  // loss_cap: rows of the per-row loss buffer
@@ -73,12 +74,13 @@ constexpr int kSortBuckets = 2048;  // power of two
 __host__ __device__ inline size_t sort_scratch_bytes(int n) { return 8u * (size_t)round_up(n, 2) + 4u * kSortBuckets; }
 
 // Dynamic shared memory of one fit.  vreg: second moments of W1 live in registers.
+// pipe: the pipelined schedule (three row buffers, two activation buffers).
 __host__ __device__ inline size_t fit_smem_bytes(int d, int dp, int Hs, int C, int CS, int TB, int order_bytes,
-                                                 int loss_cap, int n_sort, bool vreg) {
+                                                 int loss_cap, int n_sort, bool vreg, bool pipe = false) {
   const Layout L(d, Hs, C, CS);
   size_t bytes = 4u * (size_t)(2 * L.PS + (vreg ? L.PT : L.PS));
-  bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + 8u * TB + 4u * (size_t)TB * CS;
-  const size_t xa = 8u * (size_t)TB * dp + 4u * (size_t)TB * (Hs + 4);
+  bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + (pipe ? 12u : 8u) * TB + 4u * (size_t)TB * CS;
+  const size_t xa = (pipe ? 12u : 8u) * (size_t)TB * dp + (pipe ? 8u : 4u) * (size_t)TB * (Hs + 4);
   const size_t keys = sort_scratch_bytes(n_sort);
   return bytes + (xa > keys ? xa : keys);
 }

@@ -10,8 +10,17 @@
 namespace bbo {
 
 template <>
-const void* fast_fit_kernel<BBO_HSC>(bool vreg) {
+const void* fast_fit_kernel<BBO_HSC>(bool vreg, bool pipe) {
   constexpr int NT = (BBO_HSC + 31) / 32 * 32;
+#if BBO_HSC >= 128
+  constexpr int NTP = NT + 64 <= kMaxFitThreads ? NT + 64 : NT + 32;  // one or two extra warps for the output layer
+  if (pipe) {
+    if (vreg) return reinterpret_cast<const void*>(&mlp_cv_fit_kernel<kFastClasses, true, BBO_HSC, kFastDp, NTP, 1, true>);
+    return reinterpret_cast<const void*>(&mlp_cv_fit_kernel<kFastClasses, false, BBO_HSC, kFastDp, NTP, 1, true>);
+  }
+#else
+  if (pipe) return nullptr;
+#endif
   if (vreg) return reinterpret_cast<const void*>(&mlp_cv_fit_kernel<kFastClasses, true, BBO_HSC, kFastDp, NT, 1>);
   return reinterpret_cast<const void*>(&mlp_cv_fit_kernel<kFastClasses, false, BBO_HSC, kFastDp, NT, 1>);
 }

@@ -352,7 +352,7 @@ __device__ __forceinline__ void row_delta(const FitView& v, int task, int CS, co
 }
 
 // The whole fit.  CT: class count.  VR: second moments of W1 in registers.
-template <int CT, bool VR, int HSC, int DPC>
+template <int CT, bool VR, int HSC, int DPC, bool PL>
 __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, BlockShared& sh) {
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
   const int2 cf = a.fits[q];
@@ -385,10 +385,10 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   char* p = reinterpret_cast<char*>(v.M + L.PS + (VR ? L.PT : L.PS));
   v.order = reinterpret_cast<uint16_t*>(p); p += a.order_bytes;
   v.lossb = reinterpret_cast<float*>(p);    p += round_up(4 * a.loss_cap, 16);
-  v.ys = reinterpret_cast<float*>(p);       p += 8 * TB;
+  v.ys = reinterpret_cast<float*>(p);       p += (PL ? 12 : 8) * TB;   // one label buffer per row buffer
   v.D2 = reinterpret_cast<float*>(p);       p += 4 * TB * CS;
   v.Xs = reinterpret_cast<float*>(p);
-  v.A1 = v.Xs + 2 * TB * dp;
+  v.A1 = v.Xs + (PL ? 3 : 2) * TB * dp;                                 // PL: three row buffers, two of A1
   v.keys = reinterpret_cast<uint64_t*>(p);
 
   // ---- initialisation: Glorot-uniform parameters, zero moments ----
@@ -440,6 +440,8 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   const int o_first = nt >= 64 ? nt - 32 : 0;       // gb2 / b2 owners sit in the last warp, away from the unit threads
   const bool o_role = tid >= o_first && tid < o_first + CT;
   const int oo = tid - o_first;
+  const int nt_main = PL ? nt - 32 * a.extra_warps : nt;  // PL: the last warps only run the output layer
+  const int out_w0 = nt_main >> 5;
   const OutLane<CT> ol(lane);                       // output phase: lane pair = one row, each lane half the classes
   constexpr int QA = OutLane<CT>::QA;
 
@@ -457,7 +459,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   for (int e = 0; e < c.epochs; ++e) {
     build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, holdout ? 0 : vs, a.seed, rng_config, rng_fold, e, tid, nt);
     BBO_PHASE(1);
-    int buf = 0;
+    int buf = 0, abuf = 0;
     {  // first sub-tile of the epoch
       const int Bs0 = n_tr < B ? n_tr : B, nb0 = Bs0 < TB ? Bs0 : TB;
       const uint16_t* rows = v.order;
@@ -482,41 +484,23 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 #pragma unroll
       for (int o = 0; o < CT; ++o) { g2[o] = 0.f; w2[o] = unit_role ? v.W[L.oW2 + o * L.WP + tid] : 0.f; }
 
-      for (int t0 = 0; t0 < Bs; t0 += TB) {
-        const int nb = (Bs - t0) < TB ? (Bs - t0) : TB;
-        // rows of this sub-tile have landed; everyone is past the previous gW1 phase
-        cp_async_wait_all();
-        __syncthreads();
-        BBO_PHASE(2);
-        const float* xs = v.Xs + buf * TB * dp;
-        const float* ysb = v.ys + buf * TB;
-        {  // prefetch the next sub-tile of this epoch into the other buffer
-          int nt0 = t0 + TB, ns0 = s0, nBs = Bs;
-          if (nt0 >= Bs) { ns0 = s0 + B; nt0 = 0; nBs = (n_tr - ns0) < B ? (n_tr - ns0) : B; }
-          if (ns0 < n_tr) {
-            const int nnb = (nBs - nt0) < TB ? (nBs - nt0) : TB;
-            const uint16_t* rows = v.order + ns0 + nt0;
-            stage_rows_async(a, a.X, a.y, v, dp, buf ^ 1, nnb, [&](int r) { return (int)rows[r]; }, tid, nt);
-          }
-        }
-        forward_hidden(v, L, xs, d, dp, Hs, nb, tid, nt);
-        __syncthreads();
-        BBO_PHASE(3);
-
-        // ---- output layer, softmax / residual, loss derivative (lane pairs own rows) ----
-        for (int r0 = warp * 16; r0 < nb; r0 += n_warps * 16) {  // warp-uniform
+      // ---- the phases of one sub-tile; A1b: the sub-tile's buffer of hidden activations ----
+      // output layer, softmax / residual, loss derivative (lane pairs own rows), by warps w0 .. w0+nw-1
+      auto output_phase = [&](float* A1b, const float* ysb, int nb, int t0, int w0, int nw) {
+        FitView vv = v;
+        vv.A1 = A1b;
+        for (int r0 = (warp - w0) * 16; r0 < nb; r0 += nw * 16) {  // warp-uniform
           const int brow = r0 + (lane >> 1);
           const bool act = brow < nb;
           float z[QA];
-          output_logits<CT>(v, L, H, ol, act ? brow : nb - 1, z);
-          row_delta<CT>(v, a.task, CS, ol, z, act ? ysb[brow] : 0.f, brow, act, invB, want_loss, t0 + brow);
+          output_logits<CT>(vv, L, H, ol, act ? brow : nb - 1, z);
+          row_delta<CT>(vv, a.task, CS, ol, z, act ? ysb[brow] : 0.f, brow, act, invB, want_loss, t0 + brow);
         }
-        __syncthreads();
-        BBO_PHASE(4);
-
-        // ---- hidden unit tid: gW2[tid][:], delta1[:, tid] in place over A1, gb1[tid]; b ascending ----
+      };
+      // hidden unit tid: gW2[tid][:], delta1[:, tid] in place over A1, gb1[tid]; b ascending
+      auto unit_phase = [&](float* A1b, int nb) {
         if (unit_role) {
-          float* ap = v.A1 + tid;
+          float* ap = A1b + tid;
           constexpr int C4 = (CT + 3) / 4;
           int b = 0;
           for (; b + 4 <= nb; b += 4) {  // four rows at a time: loads first, then four independent delta1 chains
@@ -561,16 +545,15 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           }
         }
         if (o_role) for (int b = 0; b < nb; ++b) gb2 = __fadd_rn(gb2, v.D2[b * CS + oo]);
-        __syncthreads();
-        BBO_PHASE(5);
-
-        // ---- gW1 tile: rows k0..k0+7, columns jA..jA+3 and jB..jB+3, b ascending ----
+      };
+      // gW1 tile: rows k0..k0+7, columns jA..jA+3 and jB..jB+3, b ascending
+      auto gw1_phase = [&](const float* xs, const float* A1b, int nb) {
         if (has_tile) {
           // Two operand sets in flight: the loads of row b + 1 are issued before the multiply-adds
           // of row b, so a warp does not sit out the shared-memory latency once per row.
           const float* xp = xs + k0;
-          const float* da = v.A1 + jA;
-          const float* db = v.A1 + jB;
+          const float* da = A1b + jA;
+          const float* db = A1b + jB;
           GradOperands opA, opB;
           opA.load(xp, da, db, 0, dp, L.WP);
           int b = 0;
@@ -583,8 +566,82 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           }
           if (b < nb) opA.accumulate(g1);
         }
-        buf ^= 1;
-        BBO_PHASE(6);
+      };
+      // prefetch of the sub-tile that follows (t0 of step s0) in this epoch into row buffer `into`
+      auto prefetch_next = [&](int t0, int into) {
+        int nt0 = t0 + TB, ns0 = s0, nBs = Bs;
+        if (nt0 >= Bs) { ns0 = s0 + B; nt0 = 0; nBs = (n_tr - ns0) < B ? (n_tr - ns0) : B; }
+        if (ns0 < n_tr) {
+          const int nnb = (nBs - nt0) < TB ? (nBs - nt0) : TB;
+          const uint16_t* rows = v.order + ns0 + nt0;
+          stage_rows_async(a, a.X, a.y, v, dp, into, nnb, [&](int r) { return (int)rows[r]; }, tid, nt);
+        }
+      };
+
+      if constexpr (!PL) {
+        for (int t0 = 0; t0 < Bs; t0 += TB) {
+          const int nb = (Bs - t0) < TB ? (Bs - t0) : TB;
+          // rows of this sub-tile have landed; everyone is past the previous gW1 phase
+          cp_async_wait_all();
+          __syncthreads();
+          BBO_PHASE(2);
+          const float* xs = v.Xs + buf * TB * dp;
+          const float* ysb = v.ys + buf * TB;
+          prefetch_next(t0, buf ^ 1);
+          forward_hidden(v, L, xs, d, dp, Hs, nb, tid, nt);
+          __syncthreads();
+          BBO_PHASE(3);
+          output_phase(v.A1, ysb, nb, t0, 0, n_warps);
+          __syncthreads();
+          BBO_PHASE(4);
+          unit_phase(v.A1, nb);
+          __syncthreads();
+          BBO_PHASE(5);
+          gw1_phase(xs, v.A1, nb);
+          buf ^= 1;
+          BBO_PHASE(6);
+        }
+      } else {
+        // Pipelined schedule: the gradient tiles of sub-tile t-1 are accumulated while the extra
+        // warps (which own no tile and no hidden unit) run the output layer of sub-tile t.  Three
+        // row buffers (t-1 for the gradient, t for the forward pass, t+1 in flight) and two
+        // activation buffers make the two independent.  Every accumulator still receives its
+        // rows in ascending order: each is owned by one thread, which visits the sub-tiles in order.
+        const int T = (Bs + TB - 1) / TB;
+        for (int i = 0; i <= T; ++i) {
+          const int t0 = i * TB;
+          const int nb = i < T ? ((Bs - t0) < TB ? (Bs - t0) : TB) : 0;
+          cp_async_wait_all();
+          __syncthreads();  // rows of sub-tile i have landed; everyone is past the unit phase of i-1
+          BBO_PHASE(2);
+          const int xb = buf, xb_prev = buf == 0 ? 2 : buf - 1, xb_next = buf == 2 ? 0 : buf + 1;
+          float* A1cur = v.A1 + abuf * TB * L.WP;
+          float* A1prev = v.A1 + (abuf ^ 1) * TB * L.WP;
+          const float* ysb = v.ys + xb * TB;
+          if (i < T) {
+            prefetch_next(t0, xb_next);
+            if (tid < nt_main) {
+              FitView vv = v;
+              vv.A1 = A1cur;
+              forward_hidden(vv, L, v.Xs + xb * TB * dp, d, dp, Hs, nb, tid, nt_main);
+            }
+          }
+          __syncthreads();
+          BBO_PHASE(3);
+          if (i < T && warp >= out_w0) output_phase(A1cur, ysb, nb, t0, out_w0, n_warps - out_w0);
+          if (i > 0) {
+            const int pnb = (Bs - (t0 - TB)) < TB ? (Bs - (t0 - TB)) : TB;
+            gw1_phase(v.Xs + xb_prev * TB * dp, A1prev, pnb);
+          }
+          __syncthreads();
+          BBO_PHASE(6);
+          if (i < T) {
+            unit_phase(A1cur, nb);
+            buf = xb_next;
+            abuf ^= 1;
+          }
+          BBO_PHASE(5);
+        }
       }
       __syncthreads();  // A1 / D2 / W reads of this step are done; step size is visible
       BBO_PHASE(7);
@@ -818,11 +875,11 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 }
 
 // One CTA per fit; blockIdx.x indexes this launch's fit list (costliest first).
-template <int CT, bool VR, int HSC, int DPC, int NTMAX, int MINB>
+template <int CT, bool VR, int HSC, int DPC, int NTMAX, int MINB, bool PL = false>
 __global__ void __launch_bounds__(NTMAX, MINB) mlp_cv_fit_kernel(const FitArgs a) {
   extern __shared__ __align__(16) float smem[];
   __shared__ BlockShared sh;
-  run_fit<CT, VR, HSC, DPC>(a, blockIdx.x, smem, sh);
+  run_fit<CT, VR, HSC, DPC, PL>(a, blockIdx.x, smem, sh);
 }
 
 }  // namespace bbo

@@ -16,11 +16,16 @@ constexpr int kMaxFitThreads = 256;  // launch bound of every fit kernel
 // Hs in [kFastHsMin, kFastHsMax] (multiples of 8).
 constexpr int kFastDp = 64, kFastClasses = 10, kFastHsMin = 56, kFastHsMax = 200;
 
+// Pipelined schedule (gradient tiles of one sub-tile overlap the output layer of the next, run by
+// extra warps): built for the fast-path widths that sit alone on an SM.
+constexpr int kPipeHsMin = 128;
+inline int pipe_extra_warps(int Hs) { return (Hs + 31) / 32 * 32 + 64 <= kMaxFitThreads ? 2 : 1; }
+
 template <int CT> const void* generic_fit_kernel(bool vreg);   // run-time strides
-template <int HSC> const void* fast_fit_kernel(bool vreg);     // compile-time strides
+template <int HSC> const void* fast_fit_kernel(bool vreg, bool pipe);  // compile-time strides; pipe: pipelined schedule
 
 // Kernel for a launch of fits with C classes, padded width Hs, padded feature count dp;
 // vreg: second moments of W1 in registers.  Null when C is out of range.
-const void* fit_kernel_for(int C, int Hs, int dp, bool vreg);
+const void* fit_kernel_for(int C, int Hs, int dp, bool vreg, bool pipe = false);
 
 }  // namespace bbo
