@@ -19,6 +19,7 @@ _LIB = os.path.join(_HERE, "libmlp_cv_oracle.so")
 
 MODE_F32 = 0
 MODE_F64 = 1
+MODE_F32_TF32_OPERANDS = 2   # experiment: operands of the two large contractions rounded to TF32
 STREAM_FOLD, STREAM_INIT, STREAM_PERM = 1, 2, 3
 SOLVER_ADAM, SOLVER_SGD = 0, 1
 METRIC_DEFAULT, METRIC_ALT = 0, 1   # accuracy / -MSE, or -NLL / -MAE

@@ -13,7 +13,9 @@
 // Kingma-Ba "efficient" form, Glorot-uniform initialisation, shuffled minibatches each
 // epoch.  Every floating-point operation on the training path has a fixed order so that
 // the float mode is reproducible bit for bit; the double mode runs the same steps in
-// binary64 and exists for gradient checks and distance-from-truth reports.
+// binary64 and exists for gradient checks and distance-from-truth reports.  A third mode is an
+// experiment, never a reference: float arithmetic with the operands of the two large contractions
+// rounded to TF32 first, to measure what tensor-core inputs would do to the scores.
 //
 // Pinned (tests/test_oracle_*.py) against: the published Philox-4x32-10 known answers, a
 // Python big-integer restatement and the inverse bijection; libm exp; torch autograd
@@ -127,6 +129,21 @@ template <> struct Fn<double> {
   static double fma_(double a, double b, double c) { return std::fma(a, b, c); }
 };
 
+// Round-to-nearest-even to the 10-bit mantissa of the TF32 tensor-core input format (inf and NaN
+// pass through).  Used only by the experiment mode that asks what such operands would do to the
+// scores; the products are still accumulated in the mode's own precision.
+inline float tf32_round(float x) {
+  uint32_t u;
+  std::memcpy(&u, &x, 4);
+  if (((u >> 23) & 0xFFu) == 0xFFu) return x;
+  u += 0xFFFu + ((u >> 13) & 1u);
+  u &= ~0x1FFFu;
+  float y;
+  std::memcpy(&y, &u, 4);
+  return y;
+}
+template <typename T> inline T tf32_operand(T x) { return (T)tf32_round((float)x); }
+
 struct Config {  // one suggested configuration, 32 bytes; same field order as the library's
   int32_t hidden, batch_size, epochs;
   float alpha, lr, beta1, beta2, eps;
@@ -135,6 +152,7 @@ struct Config {  // one suggested configuration, 32 bytes; same field order as t
 // Parameter vector layout: W1[d][H] row-major, b1[H], W2[H][C] row-major, b2[C].
 struct Shape {
   int32_t d, H, C;
+  bool tf32 = false;  // experiment mode: operands of the two large contractions rounded to TF32
   int64_t oW1() const { return 0; }
   int64_t ob1() const { return (int64_t)d * H; }
   int64_t oW2() const { return ob1() + H; }
@@ -168,8 +186,14 @@ void forward_row(const Shape& s, const T* th, const T* x, T* z1, T* a1, T* z2) {
   // z1[j] = b1[j] + sum_k x[k] W1[k][j], each sum accumulated in ascending k by fused
   // multiply-add (the k loop is outermost only so that memory is walked row by row).
   for (int32_t j = 0; j < s.H; ++j) z1[j] = b1[j];
-  for (int32_t k = 0; k < s.d; ++k)
-    for (int32_t j = 0; j < s.H; ++j) z1[j] = Fn<T>::fma_(x[k], W1[(int64_t)k * s.H + j], z1[j]);
+  if (s.tf32) {
+    for (int32_t k = 0; k < s.d; ++k)
+      for (int32_t j = 0; j < s.H; ++j)
+        z1[j] = Fn<T>::fma_(tf32_operand(x[k]), tf32_operand(W1[(int64_t)k * s.H + j]), z1[j]);
+  } else {
+    for (int32_t k = 0; k < s.d; ++k)
+      for (int32_t j = 0; j < s.H; ++j) z1[j] = Fn<T>::fma_(x[k], W1[(int64_t)k * s.H + j], z1[j]);
+  }
   for (int32_t j = 0; j < s.H; ++j) a1[j] = z1[j] > (T)0 ? z1[j] : (T)0;
   // z2[o] = b2[o] + sum_j a1[j] W2[j][o], ascending j.
   for (int32_t o = 0; o < s.C; ++o) z2[o] = b2[o];
@@ -231,10 +255,18 @@ T loss_and_grad(const Shape& s, int32_t task, T alpha, const T* th, const T* xb,
     }
   // gW1[k][j] = sum_b x[b][k] d1[b][j], every sum in ascending b.
   for (int64_t i = 0; i < (int64_t)d * H; ++i) gW1[i] = (T)0;
-  for (int32_t b = 0; b < Bs; ++b)
-    for (int32_t k = 0; k < d; ++k)
-      for (int32_t j = 0; j < H; ++j)
-        gW1[(int64_t)k * H + j] = Fn<T>::fma_(xb[(int64_t)b * d + k], d1[(size_t)b * H + j], gW1[(int64_t)k * H + j]);
+  if (s.tf32) {
+    for (int32_t b = 0; b < Bs; ++b)
+      for (int32_t k = 0; k < d; ++k)
+        for (int32_t j = 0; j < H; ++j)
+          gW1[(int64_t)k * H + j] = Fn<T>::fma_(tf32_operand(xb[(int64_t)b * d + k]), tf32_operand(d1[(size_t)b * H + j]),
+                                                gW1[(int64_t)k * H + j]);
+  } else {
+    for (int32_t b = 0; b < Bs; ++b)
+      for (int32_t k = 0; k < d; ++k)
+        for (int32_t j = 0; j < H; ++j)
+          gW1[(int64_t)k * H + j] = Fn<T>::fma_(xb[(int64_t)b * d + k], d1[(size_t)b * H + j], gW1[(int64_t)k * H + j]);
+  }
   for (int32_t j = 0; j < H; ++j) {
     T acc = (T)0;
     for (int32_t b = 0; b < Bs; ++b) acc = acc + d1[(size_t)b * H + j];
@@ -340,7 +372,7 @@ double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, 
                int32_t K, const Config& cf, uint32_t config, uint32_t fold, uint64_t seed,
                const std::vector<int32_t>& pi, int32_t trace_steps, double* trace, double* theta_out,
                int32_t solver = SOLVER_ADAM, int32_t metric = METRIC_DEFAULT, const float* Xtest = nullptr,
-               const float* ytest = nullptr, int64_t n_test = 0) {
+               const float* ytest = nullptr, int64_t n_test = 0, bool tf32 = false) {
   // Hold-out mode (Xtest given; paper sec. 6.2: the generalisation score is taken on data held
   // out from the optimisation): train on every row, in the order of the fold permutation, and
   // score the rows of (Xtest, ytest) in their own order.  `fold` then only keys the random streams.
@@ -353,6 +385,7 @@ double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, 
   const int32_t n_tr = (int32_t)train.size();
   const int32_t B = std::min(cf.batch_size, n_tr);
   Shape s{d, cf.hidden, C};
+  s.tf32 = tf32;
   const int64_t P = s.P();
   std::vector<T> th((size_t)P), m((size_t)P, (T)0), v((size_t)P, (T)0), g((size_t)P);
   init_params<T>(s, seed, config, fold, th.data());
@@ -518,6 +551,9 @@ void oracle_adam_steps(int32_t mode, int64_t P, int32_t n_steps, double lr, doub
 //   fit_config[n_fits], fit_fold[n_fits]: which fits to run (config index into configs[]).
 //   fit_scores[n_fits]; loss_trace[n_fits*trace_steps] (or null); theta_out: parameters of
 //   the LAST listed fit (or null).  n_threads <= 0: all cores; threads split fits only.
+// mode: 0 float, 1 double, 2 float with the operands of the two large contractions (X W1 and
+// X^T delta1) rounded to TF32 first -- an experiment mode that shows what tensor-core inputs would
+// do to the scores; never the reference for anything.
 // solver: 0 Adam, 1 SGD with Nesterov momentum (momentum = the configuration's beta1).
 // metric: 0 accuracy / -MSE, 1 -NLL / -MAE.
 int oracle_mlp_cv_fits_ex(int32_t mode, const float* X, const float* y, int64_t n, int32_t d, int32_t task,
@@ -544,7 +580,8 @@ int oracle_mlp_cv_fits_ex(int32_t mode, const float* X, const float* y, int64_t 
     const Config& cf = cfg[fit_config[i]];
     fit_scores[i] = mode == 1
         ? run_fit<double>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho, solver, metric)
-        : run_fit<float>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho, solver, metric);
+        : run_fit<float>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho, solver, metric,
+                         nullptr, nullptr, 0, /*tf32=*/mode == 2);
   }
   return 0;
 }
