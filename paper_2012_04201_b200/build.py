@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbbo_mlp_cv.so")
-HEADERS = ["fit_kernel.cuh", "fit_roles.cuh", "sm100_primitives.cuh", "fit_common.cuh", "aux_kernels.cuh", "device_math.cuh", "fit_launch.h",
+HEADERS = ["fit_kernel.cuh", "sm100_primitives.cuh", "fit_common.cuh", "aux_kernels.cuh", "device_math.cuh", "fit_launch.h",
            os.path.join("..", "..", "include", "bbo_mlp_cv.h")]
 CLASS_COUNTS = list(range(1, 17))
 FAST_WIDTHS = list(range(56, 201, 8))   # padded hidden widths with compile-time strides

@@ -5,7 +5,6 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -107,10 +106,7 @@ bool is_device_ptr(const void* p, int device) {
 struct Plan {
   int C, CS, dp, Hs, TB, NT, order_bytes, loss_cap, n_sort, per_sm;
   int extra_warps;  // pipelined schedule: warps added for the output layer (0 = plain schedule)
-  bool roles;       // warp-specialised schedule
-  bbo::RoleWarps rw;
   int tmem_cols;
-  bool vreg;
   size_t smem;
   const void* kernel;
 };
@@ -132,11 +128,9 @@ int kernel_occupancy(const void* kernel, int threads, size_t smem) {
 
 // Plans the launch of fits of padded width Hs.  Threads: one per gradient tile of W1 (8 rows x
 // 8 columns) and one per hidden unit.  Sub-tile height: the largest of 32, 16, 8 that fits.
-// The second moments of W1 move to registers when that lets more CTAs share an SM.
 // probe_only: skip the occupancy queries (no CUDA calls), used by the caps query.
 int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bool tracing, bool probe_only,
                 Plan* out) {
-  static const bool use_roles = [] { const char* e = std::getenv("BBO_SCHEDULE"); return !(e && e[0] == 'p'); }();
   Plan p{};
   p.C = C;
   p.CS = bbo::round_up(C, 4);
@@ -147,65 +141,30 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
   p.loss_cap = tracing ? std::min(maxB, n_tr_max) : 0;
   p.n_sort = n_tr_max;
   const int tiles = (p.dp / 8) * (Hs / 8);
-  const size_t budget_r = (size_t)smem_optin - 1024;  // static block scalars and barriers
-  if (use_roles) {
-    for (int TB = 32; TB >= 8; TB >>= 1) {
-      bbo::RoleWarps rw = bbo::role_warps(p.dp, Hs, C, TB);
-      if (rw.nG > bbo::kMaxGradWarps) break;
-      const bool wide = bbo::wide_layout(rw);
-      if (wide && !bbo::fits_wide_layout(rw)) break;
-      if (wide) rw = bbo::kWideRoleWarps;  // every warp of the fixed layout takes part in the hand-offs
-      const size_t sm = bbo::roles_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort);
-      if (sm > budget_r) continue;
-      p.TB = TB;
-      p.roles = true;
-      p.rw = rw;
-      p.NT = 32 * rw.total();
-      p.tmem_cols = rw.nG <= 4 ? 128 : 256;
-      p.smem = sm;
-      p.per_sm = 1;
-      if (!probe_only) {
-        p.kernel = bbo::roles_kernel_for(C, Hs, p.dp, wide);
-        if (!p.kernel || kernel_occupancy(p.kernel, p.NT, sm) < 1) break;
-      }
-      *out = p;
-      return BBO_OK;
-    }
-    p.roles = false;
-  }
   p.NT = bbo::round_up(std::max(std::max(tiles, Hs), 32), 32);
   if (p.NT > bbo::kMaxFitThreads) return BBO_ERR_UNSUPPORTED;
+  p.tmem_cols = tiles <= 128 ? 128 : 256;  // 128 columns per group of four tile-owner warps
   const size_t budget = (size_t)smem_optin - 256;  // static block scalars
   for (int TB = 32; TB >= 8; TB >>= 1) {
-    const size_t plain = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, false);
-    const size_t lean = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
-    if (lean > budget) continue;
+    const size_t plain = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort);
+    if (plain > budget) continue;
     p.TB = TB;
+    p.smem = plain;
+    p.per_sm = 1;
     if (probe_only) {
-      p.vreg = plain > budget;
-      p.smem = p.vreg ? lean : plain;
-      p.per_sm = 1;
       *out = p;
       return BBO_OK;
     }
-    const void* k_plain = bbo::fit_kernel_for(C, Hs, p.dp, false);
-    const void* k_lean = bbo::fit_kernel_for(C, Hs, p.dp, true);
-    if (!k_plain || !k_lean) return BBO_ERR_UNSUPPORTED;
-    const int occ_plain = plain <= budget ? kernel_occupancy(k_plain, p.NT, plain) : 0;
-    const int occ_lean = kernel_occupancy(k_lean, p.NT, lean);
-    if (occ_plain < 1 && occ_lean < 1) continue;
-    p.vreg = occ_lean > occ_plain;
-    p.smem = p.vreg ? lean : plain;
-    p.per_sm = p.vreg ? occ_lean : occ_plain;
-    p.kernel = p.vreg ? k_lean : k_plain;
+    p.kernel = bbo::fit_kernel_for(C, Hs, p.dp);
+    if (!p.kernel) return BBO_ERR_UNSUPPORTED;
+    p.per_sm = kernel_occupancy(p.kernel, p.NT, plain);
+    if (p.per_sm < 1) continue;
     // Pipelined schedule: where the fit sits alone on its SM anyway and batches span several
     // sub-tiles, two extra warps run the output layer of one sub-tile under the gradient tiles of
-    // the previous one.  It needs a third row buffer and a second activation buffer, and pays
-    // only with all moments in shared memory and both extra warps (measured: +7 % to +15 % for
-    // widths 128..168, nothing or a loss beyond), so it is taken only then.
-    if (TB == 32 && p.per_sm == 1 && !p.vreg && Hs >= bbo::kPipeHsMin && maxB > TB && bbo::pipe_extra_warps(Hs) == 2) {
-      const void* k = bbo::fit_kernel_for(C, Hs, p.dp, false, true);
-      const size_t sm = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, false, true);
+    // the previous one.  It needs a third row buffer and a second activation buffer.
+    if (TB == 32 && p.per_sm == 1 && Hs >= bbo::kPipeHsMin && maxB > TB && bbo::pipe_extra_warps(Hs) == 2) {
+      const void* k = bbo::fit_kernel_for(C, Hs, p.dp, true);
+      const size_t sm = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
       if (k && sm <= budget && kernel_occupancy(k, p.NT + 64, sm) >= 1) {
         p.extra_warps = 2;
         p.NT += 64;
@@ -236,7 +195,6 @@ struct FitBuffers {  // device scratch of one evaluation
   const int32_t* pi;
   float* trace;
   float* keep_theta;
-  int32_t* status;  // set by a fit whose bounded device-side wait ran out
 };
 
 // Orders the fits for launch.  Grids are dispatched in launch order, so the fits are first cut
@@ -323,8 +281,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     a.n = n; a.d = d; a.dp = g.plan.dp; a.C = C; a.CS = g.plan.CS; a.K = K; a.task = task;
     a.Hs = g.plan.Hs; a.TB = g.plan.TB; a.trace_steps = trace_steps; a.loss_cap = g.plan.loss_cap;
     a.order_bytes = g.plan.order_bytes; a.seed = seed;
-    a.nG = g.plan.rw.nG; a.nH = g.plan.rw.nH; a.nO = g.plan.rw.nO; a.nU = g.plan.rw.nU;
-    a.tmem_cols = g.plan.tmem_cols; a.status = buf.status;
+    a.tmem_cols = g.plan.tmem_cols;
     cudaStream_t s = side ? env.aux[gi % env.n_aux] : env.main;
     void* kargs[] = {&a};
     // groups of different width may share one kernel instance: its limit is per launch
@@ -536,7 +493,7 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
   LaunchEnv env;
   env.smem_optin = h->smem_optin; env.main = s; env.aux = h->aux; env.n_aux = kAuxStreams;
   env.fork = h->fork; env.join = h->join;
-  FitBuffers buf{h->configs.p, h->fits.p, h->fold_scores.p, h->pi.p, trace, keep, h->misc.p + 3};
+  FitBuffers buf{h->configs.p, h->fits.p, h->fold_scores.p, h->pi.p, trace, keep};
   BBO_CUDA(h, cudaEventRecord(h->evf0, s));
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, h->opt.trace_steps, maxB,
@@ -548,10 +505,7 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
   BBO_CUDA(h, cudaGetLastError());
   ++launches;
   BBO_CUDA(h, cudaEventRecord(h->ev1, s));
-  int32_t timed_out = 0;
-  BBO_CUDA(h, cudaMemcpyAsync(&timed_out, h->misc.p + 3, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
   BBO_CUDA(h, cudaStreamSynchronize(s));
-  if (timed_out != 0) return BBO_ERR_TIMEOUT;
   BBO_CUDA(h, cudaEventElapsedTime(&h->last_ms, h->ev0, h->ev1));
   BBO_CUDA(h, cudaEventElapsedTime(&h->last_fit_ms, h->evf0, h->evf1));
   h->last_launches = launches;
@@ -858,17 +812,13 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
   LaunchEnv env;  // no side streams: creating them would be a resource allocation
   env.smem_optin = sd.smem_optin;
   env.main = s;
-  FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr, misc + 3};
+  FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr};
   int launches = 0;
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, 0, BBO_SOLVER_ADAM,
                        BBO_METRIC_DEFAULT, HoldoutRows{}, &launches, &cuda_err);
   if (rc != BBO_OK) return rc;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(fold_scores, n_configs, K, out_scores);
-  int32_t timed_out = 0;
-  if (cudaGetLastError() != cudaSuccess ||
-      cudaMemcpyAsync(&timed_out, misc + 3, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-      cudaStreamSynchronize(s) != cudaSuccess)
-    return BBO_ERR_CUDA;
-  return timed_out != 0 ? BBO_ERR_TIMEOUT : BBO_OK;
+  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return BBO_ERR_CUDA;
+  return BBO_OK;
 }

@@ -36,9 +36,7 @@ struct FitArgs {
   int32_t metric;        // 0 accuracy / -MSE, 1 -NLL / -MAE
   int32_t trace_steps, loss_cap;  // loss_cap: rows of the per-row loss buffer
   int32_t order_bytes;   // bytes reserved for the epoch order (uint16 per training row)
-  int32_t nG, nH, nO, nU; // warp-specialised schedule: warps of the gradient / hidden / output / unit roles
-  int32_t tmem_cols;     // warp-specialised schedule: tensor-memory columns of the CTA (power of two)
-  int32_t* status;       // warp-specialised schedule: set to 1 by a fit whose bounded wait ran out
+  int32_t tmem_cols;     // tensor-memory columns of the CTA (power of two): home of the W1 moments
   uint64_t seed;
 };
 
@@ -76,35 +74,14 @@ constexpr int kSortBuckets = 2048;  // power of two
 // Scratch of the in-kernel permutation: one 64-bit key per element plus the bucket counters.
 __host__ __device__ inline size_t sort_scratch_bytes(int n) { return 8u * (size_t)round_up(n, 2) + 4u * kSortBuckets; }
 
-// Dynamic shared memory of one fit.  vreg: second moments of W1 live in registers.
+// Dynamic shared memory of one fit (the moments of W1 live in tensor memory, not here).
 // pipe: the pipelined schedule (three row buffers, two activation buffers).
 __host__ __device__ inline size_t fit_smem_bytes(int d, int dp, int Hs, int C, int CS, int TB, int order_bytes,
-                                                 int loss_cap, int n_sort, bool vreg, bool pipe = false) {
-  const Layout L(d, Hs, C, CS);
-  size_t bytes = 4u * (size_t)(2 * L.PS + (vreg ? L.PT : L.PS));
-  bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + (pipe ? 12u : 8u) * TB + 4u * (size_t)TB * CS;
-  const size_t xa = (pipe ? 12u : 8u) * (size_t)TB * dp + (pipe ? 8u : 4u) * (size_t)TB * (Hs + 4);
-  const size_t keys = sort_scratch_bytes(n_sort);
-  return bytes + (xa > keys ? xa : keys);
-}
-
-// Warp-specialised schedule (fit_roles.cuh): hidden units per thread of the unit role (as many as
-// the register budget allows: each unit keeps its C output weights and their gradients in registers).
-__host__ __device__ constexpr int units_per_thread(int C) { return C <= 10 ? 4 : 2; }
-__host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
-// Depth of the buffer rings.
-constexpr int kNX = 4;  // row buffers: t+1 in flight / t forward / t-1, t-2 waiting for the gradient
-constexpr int kNA = 3;  // activation buffers: H writes t+1, O/U work on t, G reads t-1
-constexpr int kND = 2;  // loss-derivative buffers
-
-// Shared memory of one fit under this schedule.
-__host__ __device__ inline size_t roles_smem_bytes(int d, int dp, int Hs, int C, int CS, int TB, int order_bytes, int loss_cap,
-                                                   int n_sort) {
+                                                 int loss_cap, int n_sort, bool pipe = false) {
   const Layout L(d, Hs, C, CS);
   size_t bytes = 4u * (size_t)(L.PS + 2 * L.PT);
-  bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + 4u * (size_t)kND * TB * CS;
-  bytes = (bytes + 127) / 128 * 128;
-  const size_t xa = 4u * (size_t)kNX * TB * dp + 4u * (size_t)kNA * TB * (Hs + 4);
+  bytes += (size_t)order_bytes + (size_t)round_up(4 * loss_cap, 16) + (pipe ? 12u : 8u) * TB + 4u * (size_t)TB * CS;
+  const size_t xa = (pipe ? 12u : 8u) * (size_t)TB * dp + (pipe ? 8u : 4u) * (size_t)TB * (Hs + 4);
   const size_t keys = sort_scratch_bytes(n_sort);
   return bytes + (xa > keys ? xa : keys);
 }

@@ -22,8 +22,10 @@
 //           softmax and loss derivative in the same lanes (two shuffles per scan)
 //   unit    one thread per hidden unit j: gW2[j][:], delta1[:, j] (in place over A1), gb1[j]
 //   gW1     8x8 register tiles that persist across sub-tiles, b ascending; the owner applies
-//           the L2 term and Adam to exactly its elements (second moments of W1 may stay in
-//           the owner's registers for the whole fit)
+//           the L2 term and Adam to exactly its elements.  The first and second moments of W1
+//           live in tensor memory: each owner thread stores and reloads its own 128 words once
+//           per step (tcgen05.st / tcgen05.ld), which leaves shared memory to the parameters
+//           and the buffers and lets several fits share an SM
 // HSC / DPC: compile-time Hs / dp (0 = taken from the arguments) so that every shared-memory
 // access of the hot loops is base + immediate.
 #pragma once
@@ -32,6 +34,7 @@
 
 #include "device_math.cuh"
 #include "fit_common.cuh"
+#include "sm100_primitives.cuh"
 
 // Optional phase timers (compile with -DBBO_PHASE_TIMERS): thread 0 accumulates clock64 deltas
 // per phase, as seen after the barrier that ends the phase, and block 0 of each launch prints
@@ -48,7 +51,7 @@
 namespace bbo {
 
 struct FitView {  // per-fit pointers into shared memory
-  float *W, *M, *V;     // V is biased so that V[off] is valid for off >= ob1 when W1's v is in registers
+  float *W, *M, *V;     // M, V hold the moments of b1, W2, b2 only and are biased: M[off], V[off] are valid for off >= ob1
   uint16_t* order;
   float *lossb, *ys, *D2, *Xs, *A1;
   uint64_t* keys;
@@ -271,6 +274,7 @@ struct BlockShared {  // block-wide scalars
   int correct;
   float sq;
   float red[32];
+  uint32_t tmem_base;  // tensor-memory allocation of the CTA
 #ifdef BBO_PHASE_TIMERS
   long long phase[12];
 #endif
@@ -351,8 +355,8 @@ __device__ __forceinline__ void row_delta(const FitView& v, int task, int CS, co
   }
 }
 
-// The whole fit.  CT: class count.  VR: second moments of W1 in registers.
-template <int CT, bool VR, int HSC, int DPC, bool PL>
+// The whole fit.  CT: class count.  PL: pipelined schedule (extra warps for the output layer).
+template <int CT, int HSC, int DPC, bool PL>
 __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, BlockShared& sh) {
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
   const int2 cf = a.fits[q];
@@ -380,9 +384,9 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   BBO_PHASE_BEGIN();
   FitView v;
   v.W = smem;
-  v.M = v.W + L.PS;
-  v.V = VR ? (v.M + L.PS - L.ob1) : (v.M + L.PS);
-  char* p = reinterpret_cast<char*>(v.M + L.PS + (VR ? L.PT : L.PS));
+  v.M = v.W + L.PS - L.ob1;
+  v.V = v.M + L.PT;
+  char* p = reinterpret_cast<char*>(v.W + L.PS + 2 * L.PT);
   v.order = reinterpret_cast<uint16_t*>(p); p += a.order_bytes;
   v.lossb = reinterpret_cast<float*>(p);    p += round_up(4 * a.loss_cap, 16);
   v.ys = reinterpret_cast<float*>(p);       p += (PL ? 12 : 8) * TB;   // one label buffer per row buffer
@@ -392,11 +396,11 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   v.keys = reinterpret_cast<uint64_t*>(p);
 
   // ---- initialisation: Glorot-uniform parameters, zero moments ----
-  {
-    const int n_zero = 2 * L.PS + (VR ? L.PT : L.PS);
-    for (int i = tid; i < n_zero; i += nt) v.W[i] = 0.f;
-  }
+  for (int i = tid; i < L.PS + 2 * L.PT; i += nt) v.W[i] = 0.f;
+  if (warp == 0) tmem_alloc(&sh.tmem_base, (uint32_t)a.tmem_cols);
+  tmem_fence_before_sync();
   __syncthreads();
+  tmem_fence_after_sync();
   {
     const float bound1 = __fsqrt_rn(__fdiv_rn(6.0f, (float)(d + H)));
     const float bound2 = __fsqrt_rn(__fdiv_rn(6.0f, (float)(H + CT)));
@@ -436,6 +440,19 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   const bool has_tile = tid < KG * JG8;            // gW1 tile owner (host guarantees KG*JG8 <= nt)
   const int kg = has_tile ? tid / JG8 : 0, jg = has_tile ? tid - kg * JG8 : 0;
   const int k0 = kg << 3, jA = jg << 2, jB = (jg + JG8) << 2;
+  // Tensor-memory home of this thread's W1 moments.  A warp reaches the 32 lanes of its quarter
+  // (warp index mod 4); every group of four tile-owner warps gets 128 columns: first moments of
+  // tile row i in columns 8 i .. 8 i + 7, second moments in 64 + 8 i ..
+  const bool tile_warp = warp < ((KG * JG8 + 31) >> 5);
+  const uint32_t tm = sh.tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + 128u * (uint32_t)(warp >> 2);
+  if (tile_warp) {
+    float zero16[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) zero16[i] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tmem_store16(tm + 16u * i, zero16);
+    tmem_wait_stores();
+  }
   const bool unit_role = tid < H;                   // hidden unit tid: W2 column, b1, delta1 column
   const int o_first = nt >= 64 ? nt - 32 : 0;       // gb2 / b2 owners sit in the last warp, away from the unit threads
   const bool o_role = tid >= o_first && tid < o_first + CT;
@@ -450,11 +467,6 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   const uint32_t eps_safe = adam_eps_safe(eps);
   double p1 = 1.0, p2 = 1.0;  // running beta^t (thread 0 only)
   int step_no = 0;
-  float v1[8][8];             // second moments of this thread's W1 tile (VR only)
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) v1[i][j] = 0.f;
 
   for (int e = 0; e < c.epochs; ++e) {
     build_epoch_order(v.keys, reinterpret_cast<uint32_t*>(sh.red), v.order, a.pi, n_tr, vb, holdout ? 0 : vs, a.seed, rng_config, rng_fold, e, tid, nt);
@@ -669,88 +681,64 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       // ---- L2 term and Adam, by the owner of each gradient ----
       const float step = sh.step[step_no & 1];
       const bool sgd = a.solver == 1;
-      if (has_tile && sgd) {
+      if (tile_warp) {
+        // Every lane of a tile-owner warp walks the eight tile rows, two at a time (the
+        // tensor-memory accesses are warp-wide); lanes without a tile, and rows k >= d, touch only
+        // their own moments.  Two rows give sixteen independent update chains, which is what
+        // keeps a lone warp's pipeline busy; the moments of the next pair are requested before
+        // the current pair is updated.
+        uint32_t mr[2][16], vr[2][16];
+        auto request = [&](int pr, int buf) {
+          tmem_load16_issue(tm + 16u * pr, mr[buf]);
+          tmem_load16_issue(tm + 64u + 16u * pr, vr[buf]);
+        };
+        request(0, 0);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int k = k0 + i;
-          if (k < d) {
-            const int offA = L.oW1 + k * Hs + jA, offB = L.oW1 + k * Hs + jB;
-            const float4 wA = *reinterpret_cast<float4*>(v.W + offA), wB = *reinterpret_cast<float4*>(v.W + offB);
-            const float4 mA = *reinterpret_cast<float4*>(v.M + offA), mB = *reinterpret_cast<float4*>(v.M + offB);
-            float w8[8] = {wA.x, wA.y, wA.z, wA.w, wB.x, wB.y, wB.z, wB.w};
-            float m8[8] = {mA.x, mA.y, mA.z, mA.w, mB.x, mB.y, mB.z, mB.w};
-            float g8[8];
+        for (int pr = 0; pr < 4; ++pr) {
+          const int i0 = 2 * pr;
+          const bool live0 = has_tile && (k0 + i0) < d, live1 = has_tile && (k0 + i0 + 1) < d;
+          const int offA = L.oW1 + (k0 + i0) * Hs + jA, offB = L.oW1 + (k0 + i0) * Hs + jB;
+          float w16[16];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) g8[j] = __fmaf_rn(aB, w8[j], g1[i][j]);
-            sgd_group<8>(w8, m8, g8, c.lr, beta1);
-            *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
-            *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
-            *reinterpret_cast<float4*>(v.M + offA) = make_float4(m8[0], m8[1], m8[2], m8[3]);
-            *reinterpret_cast<float4*>(v.M + offB) = make_float4(m8[4], m8[5], m8[6], m8[7]);
-          }
-        }
-      } else if (has_tile) {
-        uint32_t redo = 0u;  // rows of the tile whose fast update could not be certified
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int k = k0 + i;
-          if (k < d) {
-            const int offA = L.oW1 + k * Hs + jA, offB = L.oW1 + k * Hs + jB;
-            const float4 wA = *reinterpret_cast<float4*>(v.W + offA), wB = *reinterpret_cast<float4*>(v.W + offB);
-            const float4 mA = *reinterpret_cast<float4*>(v.M + offA), mB = *reinterpret_cast<float4*>(v.M + offB);
-            float w8[8] = {wA.x, wA.y, wA.z, wA.w, wB.x, wB.y, wB.z, wB.w};
-            float m8[8] = {mA.x, mA.y, mA.z, mA.w, mB.x, mB.y, mB.z, mB.w};
-            float v8[8], g8[8];
-            if (VR) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j) v8[j] = v1[i][j];
-            } else {
-              const float4 vA = *reinterpret_cast<float4*>(v.V + offA), vB = *reinterpret_cast<float4*>(v.V + offB);
-              v8[0] = vA.x; v8[1] = vA.y; v8[2] = vA.z; v8[3] = vA.w; v8[4] = vB.x; v8[5] = vB.y; v8[6] = vB.z; v8[7] = vB.w;
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) g8[j] = __fmaf_rn(aB, w8[j], g1[i][j]);
-            const uint32_t safe = adam_group_fast<8>(w8, m8, v8, g8, beta1, beta2, omb1, omb2, step, eps, eps_safe);
-            if (safe) {
-              *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
-              *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
-            } else {
-              redo |= 1u << i;
-            }
-            *reinterpret_cast<float4*>(v.M + offA) = make_float4(m8[0], m8[1], m8[2], m8[3]);
-            *reinterpret_cast<float4*>(v.M + offB) = make_float4(m8[4], m8[5], m8[6], m8[7]);
-            if (VR) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j) v1[i][j] = v8[j];
-            } else {
-              *reinterpret_cast<float4*>(v.V + offA) = make_float4(v8[0], v8[1], v8[2], v8[3]);
-              *reinterpret_cast<float4*>(v.V + offB) = make_float4(v8[4], v8[5], v8[6], v8[7]);
-            }
-          }
-        }
-        if (redo) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            if (redo & (1u << i)) {
-              const int offA = L.oW1 + (k0 + i) * Hs + jA, offB = L.oW1 + (k0 + i) * Hs + jB;
+          for (int j = 0; j < 16; ++j) w16[j] = 0.f;
+          auto load_w = [&]() {
+            if (live0) {
               const float4 wA = *reinterpret_cast<float4*>(v.W + offA), wB = *reinterpret_cast<float4*>(v.W + offB);
-              const float4 mA = *reinterpret_cast<float4*>(v.M + offA), mB = *reinterpret_cast<float4*>(v.M + offB);
-              float w8[8] = {wA.x, wA.y, wA.z, wA.w, wB.x, wB.y, wB.z, wB.w};
-              const float m8[8] = {mA.x, mA.y, mA.z, mA.w, mB.x, mB.y, mB.z, mB.w};
-              float v8[8];
-              if (VR) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v8[j] = v1[i][j];
-              } else {
-                const float4 vA = *reinterpret_cast<float4*>(v.V + offA), vB = *reinterpret_cast<float4*>(v.V + offB);
-                v8[0] = vA.x; v8[1] = vA.y; v8[2] = vA.z; v8[3] = vA.w; v8[4] = vB.x; v8[5] = vB.y; v8[6] = vB.z; v8[7] = vB.w;
-              }
-              adam_params_ieee<8>(w8, m8, v8, step, eps);
-              *reinterpret_cast<float4*>(v.W + offA) = make_float4(w8[0], w8[1], w8[2], w8[3]);
-              *reinterpret_cast<float4*>(v.W + offB) = make_float4(w8[4], w8[5], w8[6], w8[7]);
+              w16[0] = wA.x; w16[1] = wA.y; w16[2] = wA.z; w16[3] = wA.w; w16[4] = wB.x; w16[5] = wB.y; w16[6] = wB.z; w16[7] = wB.w;
             }
+            if (live1) {
+              const float4 wA = *reinterpret_cast<float4*>(v.W + offA + Hs), wB = *reinterpret_cast<float4*>(v.W + offB + Hs);
+              w16[8] = wA.x; w16[9] = wA.y; w16[10] = wA.z; w16[11] = wA.w; w16[12] = wB.x; w16[13] = wB.y; w16[14] = wB.z; w16[15] = wB.w;
+            }
+          };
+          load_w();
+          tmem_wait_loads16(mr[pr & 1], vr[pr & 1]);
+          if (pr + 1 < 4) request(pr + 1, (pr + 1) & 1);
+          float m16[16], v16[16], g16[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            m16[j] = __uint_as_float(mr[pr & 1][j]); v16[j] = __uint_as_float(vr[pr & 1][j]);
+            g16[j] = __fmaf_rn(aB, w16[j], g1[i0 + (j >> 3)][j & 7]);
           }
+          if (sgd) {
+            sgd_group<16>(w16, m16, g16, c.lr, beta1);
+          } else if (!adam_group_fast<16>(w16, m16, v16, g16, beta1, beta2, omb1, omb2, step, eps, eps_safe)) {
+            // not certified: redo the parameter update from the stored weights with the IEEE routines
+            load_w();
+            adam_params_ieee<16>(w16, m16, v16, step, eps);
+          }
+          if (live0) {
+            *reinterpret_cast<float4*>(v.W + offA) = make_float4(w16[0], w16[1], w16[2], w16[3]);
+            *reinterpret_cast<float4*>(v.W + offB) = make_float4(w16[4], w16[5], w16[6], w16[7]);
+          }
+          if (live1) {
+            *reinterpret_cast<float4*>(v.W + offA + Hs) = make_float4(w16[8], w16[9], w16[10], w16[11]);
+            *reinterpret_cast<float4*>(v.W + offB + Hs) = make_float4(w16[12], w16[13], w16[14], w16[15]);
+          }
+          tmem_store16(tm + 16u * pr, m16);
+          tmem_store16(tm + 64u + 16u * pr, v16);
         }
+        tmem_wait_stores();
       }
       if (unit_role) {
         float wu[CT + 1], mu[CT + 1], vu[CT + 1], gu[CT + 1], wold[CT + 1];
@@ -872,14 +860,17 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     for (int i = tid; i < n2; i += nt) a.keep_theta[n1 + H + i] = v.W[L.oW2 + (i % CT) * L.WP + (i / CT)];
     for (int i = tid; i < CT; i += nt) a.keep_theta[n1 + H + n2 + i] = v.W[L.ob2 + i];
   }
+  tmem_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(sh.tmem_base, (uint32_t)a.tmem_cols);
 }
 
 // One CTA per fit; blockIdx.x indexes this launch's fit list (costliest first).
-template <int CT, bool VR, int HSC, int DPC, int NTMAX, int MINB, bool PL = false>
+template <int CT, int HSC, int DPC, int NTMAX, int MINB, bool PL = false>
 __global__ void __launch_bounds__(NTMAX, MINB) mlp_cv_fit_kernel(const FitArgs a) {
   extern __shared__ __align__(16) float smem[];
   __shared__ BlockShared sh;
-  run_fit<CT, VR, HSC, DPC, PL>(a, blockIdx.x, smem, sh);
+  run_fit<CT, HSC, DPC, PL>(a, blockIdx.x, smem, sh);
 }
 
 }  // namespace bbo

@@ -21,38 +21,17 @@ constexpr int kFastDp = 64, kFastClasses = 10, kFastHsMin = 56, kFastHsMax = 200
 constexpr int kPipeHsMin = 128;
 inline int pipe_extra_warps(int Hs) { return (Hs + 31) / 32 * 32 + 64 <= kMaxFitThreads ? 2 : 1; }
 
-// Warp-specialised schedule: warps per role for a fit of padded width Hs on dp padded features,
-// C classes, sub-tiles of TB rows.  G: one thread per 8x8 tile of W1; H: one thread per 8x8 tile
-// of a sub-tile's activations; O: a lane pair per row, sixteen rows per warp; U: one
-// thread per group of units_per_thread(C) hidden units plus C threads for the output biases.
-struct RoleWarps {
-  int nG, nH, nO, nU;
-  constexpr int total() const { return nG + nH + nO + nU; }
-};
-constexpr RoleWarps role_warps(int dp, int Hs, int C, int TB) {
-  return RoleWarps{ceil_div((dp / 8) * (Hs / 8), 32), ceil_div(((TB + 7) / 8) * (Hs / 8), 32), TB > 16 ? 2 : 1,
-                   ceil_div(Hs / units_per_thread(C) + C, 32)};
-}
-constexpr int kMaxGradWarps = 8;    // tensor memory holds the W1 moments of at most eight G warps
-// Up to twelve warps the roles are packed one after the other and every thread has 168 registers.
-// Wider fits run the 512-thread layout with the roles on warp-group boundaries (8 / 4 / 2 / 2
-// warps) and the registers re-divided between the groups.
-constexpr int kCompactRoleWarps = 12;
-constexpr RoleWarps kWideRoleWarps{8, 4, 2, 2};
-constexpr bool wide_layout(const RoleWarps& r) { return r.total() > kCompactRoleWarps; }
-constexpr bool fits_wide_layout(const RoleWarps& r) {
-  return r.nG <= kWideRoleWarps.nG && r.nH <= kWideRoleWarps.nH && r.nO <= kWideRoleWarps.nO && r.nU <= kWideRoleWarps.nU;
-}
+// Resident CTAs per SM the compile-time-width instances are built for: the launch bound caps
+// their registers at 65,536 / (CTAs x threads), and shared memory admits that many (the row
+// buffers and parameters of a fit of that width, moments of W1 in tensor memory).
+constexpr int fast_threads(int Hs) { return (Hs + 31) / 32 * 32; }
+constexpr int fast_min_blocks(int Hs) { return fast_threads(Hs) <= 64 ? 4 : (fast_threads(Hs) <= 96 ? 3 : (Hs <= 176 ? 2 : 1)); }
 
-template <int CT> const void* generic_roles_kernel(bool wide);  // warp-specialised, run-time strides
-template <int HSC> const void* fast_roles_kernel();            // warp-specialised, compile-time strides (layout follows from the width)
-const void* roles_kernel_for(int C, int Hs, int dp, bool wide);
+template <int CT> const void* generic_fit_kernel();            // run-time strides
+template <int HSC> const void* fast_fit_kernel(bool pipe);     // compile-time strides; pipe: pipelined schedule
 
-template <int CT> const void* generic_fit_kernel(bool vreg);   // run-time strides
-template <int HSC> const void* fast_fit_kernel(bool vreg, bool pipe);  // compile-time strides; pipe: pipelined schedule
-
-// Kernel for a launch of fits with C classes, padded width Hs, padded feature count dp;
-// vreg: second moments of W1 in registers.  Null when C is out of range.
-const void* fit_kernel_for(int C, int Hs, int dp, bool vreg, bool pipe = false);
+// Kernel for a launch of fits with C classes, padded width Hs, padded feature count dp.
+// Null when C is out of range or the pipelined schedule is not built for the shape.
+const void* fit_kernel_for(int C, int Hs, int dp, bool pipe = false);
 
 }  // namespace bbo
