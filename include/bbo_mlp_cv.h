@@ -1,11 +1,11 @@
 /* bbo_mlp_cv.h -- C ABI of the fused MLP-Adam cross-validation library (CUDA, sm_100a).
  *
  * The library is the `evaluate(params_list) -> scores` call of the suggest-observe loop
- * (paper, Algorithm 1): for every suggested hyperparameter configuration it returns "the
- * cross validation score of a machine learning model on a dataset with a loss function"
- * (paper, sec. 2) for the model the paper's Table 1 calls MLP-adam, with the metrics acc
- * and mse of the same table, five folds in the paper's runs (sec. 6.3: 2.7 M trainings for
- * 541,440 evaluations).  Function evaluation is what the paper moves to the GPU because it
+ * (paper, Algorithm 1): for every suggested hyperparameter configuration it returns the
+ * k-fold cross-validation score of one model / dataset / metric triple, which is the function
+ * the optimizers of the paper see (sec. 2), for the model the paper's Table 1 calls MLP-adam,
+ * with the metrics acc and mse of the same table, five folds in the paper's runs (sec. 6.3:
+ * 2.7 M trainings for 541,440 evaluations).  Function evaluation is what the paper moves to the GPU because it
  * dominates run time (sec. 1, sec. 5, sec. 6.3).
  *
  * Model and training rule (the paper names the model, not its formulas; these are the
@@ -63,6 +63,15 @@ typedef enum { BBO_SOLVER_ADAM = 0, BBO_SOLVER_SGD = 1 } bbo_solver;
  * error (row sums in ascending row order; NaN maps to -inf).  Always "higher is better".    */
 typedef enum { BBO_METRIC_DEFAULT = 0, BBO_METRIC_ALT = 1 } bbo_metric;
 
+/* Arithmetic of the two large contractions (paper sec. 5 only says the MLP is "GPU-optimized").
+ * BBO_VARIANT_FP32: binary32 fused multiply-adds on the CUDA cores in one fixed order; the only
+ * variant that is built, because the score tolerance (1e-3 on accuracies whose quantum is one
+ * held-out row) needs identical predictions after tens of thousands of optimizer steps.
+ * BBO_VARIANT_TF32 names the tensor-core variant (TF32 operands, with or without a high/low
+ * operand split); the CPU checker's experiment modes show that neither keeps 99 % of the fold
+ * scores within the tolerance, so bbo_mlp_cv_create answers BBO_ERR_UNSUPPORTED for it.       */
+typedef enum { BBO_VARIANT_FP32 = 0, BBO_VARIANT_TF32 = 1 } bbo_variant;
+
 typedef enum {
   BBO_OK = 0,
   BBO_ERR_INVALID_ARG = -1, /* NULL pointer, bad size, hyperparameter or label out of range */
@@ -89,6 +98,7 @@ typedef struct {
                           gets the scores the unsplit call would give                          */
   int32_t solver;      /* a bbo_solver; 0 = Adam                                             */
   int32_t metric;      /* a bbo_metric; 0 = accuracy / minus mean squared error               */
+  int32_t variant;     /* a bbo_variant; 0 = FP32 CUDA cores (the only one built)             */
 } bbo_mlp_cv_options;
 
 /* Creates a handle bound to one device and one stream.  `opt` may be NULL (defaults).
@@ -111,6 +121,17 @@ int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out);
 int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d,
                     int32_t task, int32_t n_folds, const bbo_mlp_config* configs,
                     int32_t n_configs, uint64_t seed, float* out_scores);
+
+/* As bbo_mlp_cv_eval, with an explicit key per configuration for its random streams instead of
+ * its position in the list (paper sec. 5 deals the jobs to the GPUs in round-robin order: a
+ * caller that splits one params_list unevenly, e.g. balanced by cost, passes each entry's
+ * position in the unsplit list and gets exactly the scores of the unsplit call).
+ *   config_keys  HOST [n_configs], each in [0, 2^28); copied during the call
+ * The handle's config_index_base is ignored by this call.                                   */
+int bbo_mlp_cv_eval_keyed(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d,
+                          int32_t task, int32_t n_folds, const bbo_mlp_config* configs,
+                          const int32_t* config_keys, int32_t n_configs, uint64_t seed,
+                          float* out_scores);
 
 /* Hold-out ("generalisation") scores of the same configurations (paper, sec. 6.2: the data
  * are split into the part the optimizers see through cross-validation and a part held out to
@@ -177,7 +198,9 @@ int bbo_mlp_cv_debug_fast_math(bbo_mlp_cv* h, int32_t mode, uint64_t seed, uint6
 int bbo_mlp_cv_debug_ffma_peak(bbo_mlp_cv* h, int32_t threads_per_sm, int32_t iters, float* tflops);
 
 /* Largest shapes one call accepts on this device: rows, features, hidden width for the
- * given (d, n_classes) pair, and classes.  Any output pointer may be NULL.               */
+ * given (d, n_classes) pair, and classes.  The hidden-width and feature caps are those of a
+ * 1797-row, 5-fold problem; they shrink for longer training folds (the per-epoch sort scratch
+ * grows with the fold).  Any output pointer may be NULL.                                  */
 int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* max_n,
                           int32_t* max_d, int32_t* max_hidden, int32_t* max_classes);
 
@@ -193,7 +216,8 @@ int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* total_ms, float* fit_ms, int32_
  * whole device heap, real-time or latency-bound loops where cudaMalloc's implicit device
  * synchronisation and unbounded latency are not acceptable, and processes that have already
  * handed all free memory to another component.  It needs no handle, and it calls neither
- * cudaMalloc nor cudaFree nor any allocating library routine.
+ * cudaMalloc nor cudaFree nor any allocating library routine (what the driver itself does when
+ * a kernel is launched for the first time is described below).
  *
  * All working memory (fold permutation, device copy of the configurations, fit list,
  * per-fold scores, work counter, padded copy of X) lives in ONE fixed array of
@@ -210,11 +234,17 @@ int bbo_mlp_cv_last_timing(bbo_mlp_cv* h, float* total_ms, float* fit_ms, int32_
  *   n_classes  classification: 0 = 1 + max(y) found on the device; ignored for regression
  *   configs    HOST [n_configs]
  *
- * The first call on each device looks up the array's device address and the device's
- * limits (a one-off set-up, cached per device); make that first call before starting any
- * stream capture.  The array is shared by every call in the process and keeps the previous
- * call's contents; the call clears what has to start from zero.  Two calls that overlap on
- * the same GPU (different streams or threads) would race on it: run them one after another. */
+ * The call is synchronous: it synchronises the stream twice (after the label scan and at the
+ * end) and copies from pageable host memory, so it cannot run inside a stream capture.  The
+ * first call on each device also looks up the array's device address and the device's limits
+ * (a one-off set-up, cached per device), and the first launch of each kernel instance lets the
+ * driver load that kernel's code, which may take device memory inside the driver: a warm-up
+ * call per data shape, made while allocation is still allowed, gets both out of the way.  The
+ * array is shared by every call in the process and keeps the previous call's contents; the
+ * call clears what has to start from zero.  Two calls that overlap on the same GPU (different
+ * streams or threads) would race on it: run them one after another.
+ * bbo_mlp_cv_static_last_cuda_error returns the text of the calling thread's last CUDA error
+ * from this entry point ("" if none).                                                        */
 #define BBO_STATIC_MAX_ROWS 4096
 #define BBO_STATIC_MAX_X_FLOATS 262144
 #define BBO_STATIC_MAX_CONFIGS 4096
@@ -225,6 +255,8 @@ int bbo_mlp_cv_eval_static(void* stream, const float* X, const float* y, int64_t
                            int32_t task, int32_t n_folds, int32_t n_classes,
                            const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed,
                            float* out_scores);
+
+const char* bbo_mlp_cv_static_last_cuda_error(void);
 
 const char* bbo_mlp_cv_strerror(int code);
 /* Text of the last CUDA error seen by this handle ("" if none).  Valid until the next call. */

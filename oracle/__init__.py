@@ -20,6 +20,8 @@ _LIB = os.path.join(_HERE, "libmlp_cv_oracle.so")
 MODE_F32 = 0
 MODE_F64 = 1
 MODE_F32_TF32_OPERANDS = 2   # experiment: operands of the two large contractions rounded to TF32
+MODE_F32_BLOCKED = 3         # experiment: exact float products, summed in blocks of 8 as a matrix unit would
+MODE_F32_BLOCKED_SPLIT = 4   # experiment: the blocked order with hi/lo TF32 operand splits (three products per term)
 STREAM_FOLD, STREAM_INIT, STREAM_PERM = 1, 2, 3
 SOLVER_ADAM, SOLVER_SGD = 0, 1
 METRIC_DEFAULT, METRIC_ALT = 0, 1   # accuracy / -MSE, or -NLL / -MAE
@@ -91,6 +93,10 @@ def lib():
         L.oracle_holdout_order.argtypes = [i64, u64, i32, i32, vp]
         L.oracle_holdout_order.restype = ctypes.c_int
         L.oracle_num_procs.restype = ctypes.c_int
+        L.oracle_tf32_round.argtypes = [ctypes.c_float]
+        L.oracle_tf32_round.restype = ctypes.c_float
+        L.oracle_tf32_split.argtypes = [ctypes.c_float, vp, vp]
+        L.oracle_tf32_split.restype = None
         _lib = L
     return _lib
 
@@ -270,6 +276,18 @@ def holdout_order(n, seed, config, epoch):
     out = np.zeros(n, np.int32)
     assert lib().oracle_holdout_order(n, seed, config, epoch, _p(out)) == 0
     return out
+
+
+def tf32_round(x):
+    """Round-to-nearest-even of a float to the 10-bit mantissa of the TF32 operand format."""
+    return float(lib().oracle_tf32_round(float(x)))
+
+
+def tf32_split(x):
+    """(hi, lo) with hi = tf32_round(x), lo = tf32_round(x - hi)."""
+    hi, lo = ctypes.c_float(), ctypes.c_float()
+    lib().oracle_tf32_split(float(x), ctypes.byref(hi), ctypes.byref(lo))
+    return hi.value, lo.value
 
 
 def num_procs():

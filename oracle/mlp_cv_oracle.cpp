@@ -13,9 +13,12 @@
 // Kingma-Ba "efficient" form, Glorot-uniform initialisation, shuffled minibatches each
 // epoch.  Every floating-point operation on the training path has a fixed order so that
 // the float mode is reproducible bit for bit; the double mode runs the same steps in
-// binary64 and exists for gradient checks and distance-from-truth reports.  A third mode is an
-// experiment, never a reference: float arithmetic with the operands of the two large contractions
-// rounded to TF32 first, to measure what tensor-core inputs would do to the scores.
+// binary64 and exists for gradient checks and distance-from-truth reports.  Three further modes
+// are experiments, never references; they ask what tensor-core arithmetic in the two large
+// contractions (X W1 and X^T delta1) would do to the scores, everything else staying float:
+// operands rounded to TF32; float products summed the way a matrix unit sums them (blocks of
+// eight terms, block sums added in order); and that blocking with every operand split into a
+// TF32 high and low part and three products per term.
 //
 // Pinned (tests/test_oracle_*.py) against: the published Philox-4x32-10 known answers, a
 // Python big-integer restatement and the inverse bijection; libm exp; torch autograd
@@ -144,6 +147,34 @@ inline float tf32_round(float x) {
 }
 template <typename T> inline T tf32_operand(T x) { return (T)tf32_round((float)x); }
 
+// Experiment modes of the two large contractions (Shape::exp).
+enum : int32_t {
+  EXP_NONE = 0,
+  EXP_TF32_OPERANDS = 2,  // operands rounded to TF32, terms added one by one in the usual order
+  EXP_BLOCKED = 3,        // exact float products; terms in blocks of 8 summed from zero, block sums added in order
+  EXP_BLOCKED_SPLIT = 4   // EXP_BLOCKED with each operand split hi + lo (both TF32) and lo*hi + hi*lo + hi*hi per term
+};
+constexpr int32_t kMmaBlock = 8;
+
+// hi = tf32(x), lo = tf32(x - hi): x = hi + lo up to about 2^-21 relative.
+inline void tf32_split(float x, float* hi, float* lo) {
+  *hi = tf32_round(x);
+  *lo = tf32_round(x - *hi);
+}
+
+// One term a*b added to the block sum `acc` under an experiment mode.
+template <typename T> inline T exp_term(int32_t exp, T a, T b, T acc) {
+  if (exp == EXP_BLOCKED_SPLIT) {
+    float ah, al, bh, bl;
+    tf32_split((float)a, &ah, &al);
+    tf32_split((float)b, &bh, &bl);
+    acc = Fn<T>::fma_((T)al, (T)bh, acc);
+    acc = Fn<T>::fma_((T)ah, (T)bl, acc);
+    return Fn<T>::fma_((T)ah, (T)bh, acc);
+  }
+  return Fn<T>::fma_(a, b, acc);
+}
+
 struct Config {  // one suggested configuration, 32 bytes; same field order as the library's
   int32_t hidden, batch_size, epochs;
   float alpha, lr, beta1, beta2, eps;
@@ -152,7 +183,7 @@ struct Config {  // one suggested configuration, 32 bytes; same field order as t
 // Parameter vector layout: W1[d][H] row-major, b1[H], W2[H][C] row-major, b2[C].
 struct Shape {
   int32_t d, H, C;
-  bool tf32 = false;  // experiment mode: operands of the two large contractions rounded to TF32
+  int32_t exp = EXP_NONE;  // experiment mode of the two large contractions (never a reference)
   int64_t oW1() const { return 0; }
   int64_t ob1() const { return (int64_t)d * H; }
   int64_t oW2() const { return ob1() + H; }
@@ -186,10 +217,17 @@ void forward_row(const Shape& s, const T* th, const T* x, T* z1, T* a1, T* z2) {
   // z1[j] = b1[j] + sum_k x[k] W1[k][j], each sum accumulated in ascending k by fused
   // multiply-add (the k loop is outermost only so that memory is walked row by row).
   for (int32_t j = 0; j < s.H; ++j) z1[j] = b1[j];
-  if (s.tf32) {
+  if (s.exp == EXP_TF32_OPERANDS) {
     for (int32_t k = 0; k < s.d; ++k)
       for (int32_t j = 0; j < s.H; ++j)
         z1[j] = Fn<T>::fma_(tf32_operand(x[k]), tf32_operand(W1[(int64_t)k * s.H + j]), z1[j]);
+  } else if (s.exp == EXP_BLOCKED || s.exp == EXP_BLOCKED_SPLIT) {
+    for (int32_t j = 0; j < s.H; ++j)
+      for (int32_t k0 = 0; k0 < s.d; k0 += kMmaBlock) {
+        T part = (T)0;
+        for (int32_t k = k0; k < s.d && k < k0 + kMmaBlock; ++k) part = exp_term<T>(s.exp, x[k], W1[(int64_t)k * s.H + j], part);
+        z1[j] = z1[j] + part;
+      }
   } else {
     for (int32_t k = 0; k < s.d; ++k)
       for (int32_t j = 0; j < s.H; ++j) z1[j] = Fn<T>::fma_(x[k], W1[(int64_t)k * s.H + j], z1[j]);
@@ -255,12 +293,24 @@ T loss_and_grad(const Shape& s, int32_t task, T alpha, const T* th, const T* xb,
     }
   // gW1[k][j] = sum_b x[b][k] d1[b][j], every sum in ascending b.
   for (int64_t i = 0; i < (int64_t)d * H; ++i) gW1[i] = (T)0;
-  if (s.tf32) {
+  if (s.exp == EXP_TF32_OPERANDS) {
     for (int32_t b = 0; b < Bs; ++b)
       for (int32_t k = 0; k < d; ++k)
         for (int32_t j = 0; j < H; ++j)
           gW1[(int64_t)k * H + j] = Fn<T>::fma_(tf32_operand(xb[(int64_t)b * d + k]), tf32_operand(d1[(size_t)b * H + j]),
                                                 gW1[(int64_t)k * H + j]);
+  } else if (s.exp == EXP_BLOCKED || s.exp == EXP_BLOCKED_SPLIT) {
+    for (int32_t k = 0; k < d; ++k)
+      for (int32_t j = 0; j < H; ++j) {
+        T acc = (T)0;
+        for (int32_t b0 = 0; b0 < Bs; b0 += kMmaBlock) {
+          T part = (T)0;
+          for (int32_t b = b0; b < Bs && b < b0 + kMmaBlock; ++b)
+            part = exp_term<T>(s.exp, xb[(int64_t)b * d + k], d1[(size_t)b * H + j], part);
+          acc = acc + part;
+        }
+        gW1[(int64_t)k * H + j] = acc;
+      }
   } else {
     for (int32_t b = 0; b < Bs; ++b)
       for (int32_t k = 0; k < d; ++k)
@@ -372,7 +422,7 @@ double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, 
                int32_t K, const Config& cf, uint32_t config, uint32_t fold, uint64_t seed,
                const std::vector<int32_t>& pi, int32_t trace_steps, double* trace, double* theta_out,
                int32_t solver = SOLVER_ADAM, int32_t metric = METRIC_DEFAULT, const float* Xtest = nullptr,
-               const float* ytest = nullptr, int64_t n_test = 0, bool tf32 = false) {
+               const float* ytest = nullptr, int64_t n_test = 0, int32_t exp = EXP_NONE) {
   // Hold-out mode (Xtest given; paper sec. 6.2: the generalisation score is taken on data held
   // out from the optimisation): train on every row, in the order of the fold permutation, and
   // score the rows of (Xtest, ytest) in their own order.  `fold` then only keys the random streams.
@@ -385,7 +435,7 @@ double run_fit(const float* X, const float* y, int64_t n, int32_t d, int32_t C, 
   const int32_t n_tr = (int32_t)train.size();
   const int32_t B = std::min(cf.batch_size, n_tr);
   Shape s{d, cf.hidden, C};
-  s.tf32 = tf32;
+  s.exp = exp;
   const int64_t P = s.P();
   std::vector<T> th((size_t)P), m((size_t)P, (T)0), v((size_t)P, (T)0), g((size_t)P);
   init_params<T>(s, seed, config, fold, th.data());
@@ -551,8 +601,9 @@ void oracle_adam_steps(int32_t mode, int64_t P, int32_t n_steps, double lr, doub
 //   fit_config[n_fits], fit_fold[n_fits]: which fits to run (config index into configs[]).
 //   fit_scores[n_fits]; loss_trace[n_fits*trace_steps] (or null); theta_out: parameters of
 //   the LAST listed fit (or null).  n_threads <= 0: all cores; threads split fits only.
-// mode: 0 float, 1 double, 2 float with the operands of the two large contractions (X W1 and
-// X^T delta1) rounded to TF32 first -- an experiment mode that shows what tensor-core inputs would
+// mode: 0 float, 1 double; 2, 3, 4: the float experiment modes EXP_TF32_OPERANDS, EXP_BLOCKED,
+// EXP_BLOCKED_SPLIT of the two large contractions (X W1 and
+// X^T delta1) -- experiment modes that show what tensor-core arithmetic would
 // do to the scores; never the reference for anything.
 // solver: 0 Adam, 1 SGD with Nesterov momentum (momentum = the configuration's beta1).
 // metric: 0 accuracy / -MSE, 1 -NLL / -MAE.
@@ -581,7 +632,7 @@ int oracle_mlp_cv_fits_ex(int32_t mode, const float* X, const float* y, int64_t 
     fit_scores[i] = mode == 1
         ? run_fit<double>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho, solver, metric)
         : run_fit<float>(X, y, n, d, C, task, n_folds, cf, fit_config[i], fit_fold[i], seed, pi, trace_steps, tr, tho, solver, metric,
-                         nullptr, nullptr, 0, /*tf32=*/mode == 2);
+                         nullptr, nullptr, 0, /*exp=*/mode >= 2 ? mode : EXP_NONE);
   }
   return 0;
 }
@@ -692,6 +743,9 @@ void oracle_sgd_steps(int32_t mode, int64_t P, int32_t n_steps, double lr, doubl
   }
   for (int64_t i = 0; i < P; ++i) { theta[i] = th[i]; vel[i] = vv[i]; }
 }
+
+float oracle_tf32_round(float x) { return tf32_round(x); }
+void oracle_tf32_split(float x, float* hi, float* lo) { tf32_split(x, hi, lo); }
 
 int oracle_num_procs(void) {
 #ifdef _OPENMP

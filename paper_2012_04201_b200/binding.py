@@ -28,9 +28,11 @@ TASK_CLASSIFICATION = 0
 TASK_REGRESSION = 1
 SOLVER_ADAM, SOLVER_SGD = 0, 1
 METRIC_DEFAULT, METRIC_ALT = 0, 1
+VARIANT_FP32, VARIANT_TF32 = 0, 1
 
 EXPORTS = [
     "bbo_mlp_cv_create", "bbo_mlp_cv_eval", "bbo_mlp_cv_eval_host", "bbo_mlp_cv_eval_holdout", "bbo_mlp_cv_destroy",
+    "bbo_mlp_cv_eval_keyed", "bbo_mlp_cv_static_last_cuda_error",
     "bbo_mlp_cv_fold_scores", "bbo_mlp_cv_loss_trace", "bbo_mlp_cv_debug_theta",
     "bbo_mlp_cv_debug_indices", "bbo_mlp_cv_debug_rng", "bbo_mlp_cv_debug_exp",
     "bbo_mlp_cv_query_caps", "bbo_mlp_cv_last_timing", "bbo_mlp_cv_strerror",
@@ -41,7 +43,8 @@ EXPORTS = [
 class Options(ctypes.Structure):
     _fields_ = [("device", ctypes.c_int32), ("stream", ctypes.c_void_p), ("n_classes", ctypes.c_int32),
                 ("trace_steps", ctypes.c_int32), ("keep_theta", ctypes.c_int32),
-                ("config_index_base", ctypes.c_int32), ("solver", ctypes.c_int32), ("metric", ctypes.c_int32)]
+                ("config_index_base", ctypes.c_int32), ("solver", ctypes.c_int32), ("metric", ctypes.c_int32),
+                ("variant", ctypes.c_int32)]
 
 
 _lib = None
@@ -69,6 +72,9 @@ def load():
     L.bbo_mlp_cv_create.argtypes = [ctypes.POINTER(Options), ctypes.POINTER(vp)]
     L.bbo_mlp_cv_eval.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_eval_host.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, i32, u64, vp]
+    L.bbo_mlp_cv_eval_keyed.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, vp, i32, u64, vp]
+    L.bbo_mlp_cv_static_last_cuda_error.argtypes = []
+    L.bbo_mlp_cv_static_last_cuda_error.restype = ctypes.c_char_p
     L.bbo_mlp_cv_eval_holdout.argtypes = [vp, vp, vp, i64, vp, vp, i64, i32, i32, vp, i32, u64, vp]
     L.bbo_mlp_cv_destroy.argtypes = [vp]
     L.bbo_mlp_cv_eval_static.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, i32, u64, vp]
@@ -87,7 +93,7 @@ def load():
     L.bbo_mlp_cv_last_cuda_error.argtypes = [vp]
     L.bbo_mlp_cv_last_cuda_error.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("bbo_mlp_cv_strerror", "bbo_mlp_cv_last_cuda_error"):
+        if name not in ("bbo_mlp_cv_strerror", "bbo_mlp_cv_last_cuda_error", "bbo_mlp_cv_static_last_cuda_error"):
             getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -106,10 +112,10 @@ def _np_ptr(a):
 
 # ---- functions with the C names -------------------------------------------------------
 def bbo_mlp_cv_create(device=-1, stream=0, n_classes=0, trace_steps=0, keep_theta=0, config_index_base=0,
-                      solver=SOLVER_ADAM, metric=METRIC_DEFAULT):
+                      solver=SOLVER_ADAM, metric=METRIC_DEFAULT, variant=VARIANT_FP32):
     opt = Options(device=device, stream=stream or None, n_classes=n_classes, trace_steps=trace_steps,
                   keep_theta=int(keep_theta), config_index_base=int(config_index_base), solver=int(solver),
-                  metric=int(metric))
+                  metric=int(metric), variant=int(variant))
     h = ctypes.c_void_p()
     rc = load().bbo_mlp_cv_create(ctypes.byref(opt), ctypes.byref(h))
     if rc != BBO_OK:
@@ -122,6 +128,15 @@ def bbo_mlp_cv_eval(h, X_ptr, y_ptr, n, d, task, n_folds, configs, seed, out_ptr
     configs = np.ascontiguousarray(configs, dtype=CONFIG_DTYPE)
     return load().bbo_mlp_cv_eval(h, X_ptr, y_ptr, n, d, task, n_folds, _np_ptr(configs), configs.size,
                                   seed, out_ptr)
+
+
+def bbo_mlp_cv_eval_keyed(h, X_ptr, y_ptr, n, d, task, n_folds, configs, config_keys, seed, out_ptr):
+    """As bbo_mlp_cv_eval with one random-stream key per configuration (int32 array)."""
+    configs = np.ascontiguousarray(configs, dtype=CONFIG_DTYPE)
+    keys = np.ascontiguousarray(config_keys, dtype=np.int32)
+    assert keys.size == configs.size
+    return load().bbo_mlp_cv_eval_keyed(h, X_ptr, y_ptr, n, d, task, n_folds, _np_ptr(configs), _np_ptr(keys),
+                                        configs.size, seed, out_ptr)
 
 
 def bbo_mlp_cv_eval_host(h, X, y, task, n_folds, configs, seed, out):
@@ -149,7 +164,7 @@ class MlpCv:
     """One handle = one device, one stream, one call in flight."""
 
     def __init__(self, device=None, stream=None, n_classes=0, trace_steps=0, keep_theta=False, config_index_base=0,
-                 solver=SOLVER_ADAM, metric=METRIC_DEFAULT):
+                 solver=SOLVER_ADAM, metric=METRIC_DEFAULT, variant=VARIANT_FP32):
         import torch
 
         if not torch.cuda.is_available():
@@ -162,7 +177,7 @@ class MlpCv:
         self.stream = stream
         sptr = 0 if stream is None else int(stream.cuda_stream)
         self._h = bbo_mlp_cv_create(self.device, sptr, n_classes, trace_steps, keep_theta, config_index_base,
-                                    solver, metric)
+                                    solver, metric, variant)
         self._n_configs = self._n_folds = 0
         self.trace_steps = trace_steps
 
@@ -170,8 +185,9 @@ class MlpCv:
         if rc != BBO_OK:
             raise BboError(rc, load().bbo_mlp_cv_last_cuda_error(self._h).decode())
 
-    def eval(self, X, y, task, n_folds, configs, seed, out=None):
-        """``X`` [n, d], ``y`` [n]: float32 CUDA tensors.  Returns scores [n_configs] (CUDA)."""
+    def eval(self, X, y, task, n_folds, configs, seed, out=None, config_keys=None):
+        """``X`` [n, d], ``y`` [n]: float32 CUDA tensors.  Returns scores [n_configs] (CUDA).
+        ``config_keys``: optional int32 key per configuration for its random streams."""
         torch = self._torch
         assert X.is_cuda and y.is_cuda and X.dtype == torch.float32 and y.dtype == torch.float32
         X = X.contiguous()
@@ -181,8 +197,12 @@ class MlpCv:
             out = torch.empty(configs.size, dtype=torch.float32, device=X.device)
         if self.stream is not None:
             self.stream.wait_stream(torch.cuda.current_stream(X.device))
-        rc = bbo_mlp_cv_eval(self._h, X.data_ptr(), y.data_ptr(), X.shape[0], X.shape[1], task, n_folds,
-                             configs, seed, out.data_ptr())
+        if config_keys is None:
+            rc = bbo_mlp_cv_eval(self._h, X.data_ptr(), y.data_ptr(), X.shape[0], X.shape[1], task, n_folds,
+                                 configs, seed, out.data_ptr())
+        else:
+            rc = bbo_mlp_cv_eval_keyed(self._h, X.data_ptr(), y.data_ptr(), X.shape[0], X.shape[1], task, n_folds,
+                                       configs, config_keys, seed, out.data_ptr())
         self._check(rc)
         self._n_configs, self._n_folds = configs.size, n_folds
         return out

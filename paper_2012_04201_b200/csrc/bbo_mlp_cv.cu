@@ -23,6 +23,7 @@ namespace {
 using bbo::kMaxClasses;
 constexpr int kAuxStreams = 32;  // buckets of different hidden width overlap on these
 constexpr int kMaxRows = 16384;  // fold permutation sorts in one CTA's shared memory
+constexpr int kMaxFeatures = 16384, kMaxHidden = 8192;  // beyond any shape shared memory admits; keeps the size arithmetic in int
 
 template <typename T>
 struct DevBuf {
@@ -57,7 +58,7 @@ struct bbo_mlp_cv {
   DevBuf<bbo::Config> configs;
   DevBuf<int2> fits;
   DevBuf<float> fold_scores, trace, theta, xpad, xpad_t, hx, hy, hscores, dbg_f;
-  DevBuf<int32_t> pi, misc, dbg_i;
+  DevBuf<int32_t> pi, misc, dbg_i, keys;
   DevBuf<uint32_t> dbg_u;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr, evf0 = nullptr, evf1 = nullptr;
   cudaStream_t aux[kAuxStreams] = {};
@@ -111,9 +112,19 @@ struct Plan {
   const void* kernel;
 };
 
-// Resident CTAs per SM of a fit kernel instance (0 if it cannot launch).
-int kernel_occupancy(const void* kernel, int threads, size_t smem) {
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+// Resident CTAs per SM of a fit kernel instance (0 if it cannot launch).  The dynamic
+// shared-memory limit of an instance is always set to the device's opt-in maximum, never to the
+// size of one launch: the attribute is global to the process, and handles on different threads
+// share the instances.
+int kernel_occupancy(const void* kernel, int threads, size_t smem, int smem_optin) {
+  cudaFuncAttributes attr;
+  if (cudaFuncGetAttributes(&attr, kernel) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  const int max_dynamic = smem_optin - (int)attr.sharedSizeBytes;  // the opt-in limit covers static + dynamic
+  if ((size_t)max_dynamic < smem ||
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dynamic) != cudaSuccess ||
       cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
     cudaGetLastError();
     return 0;
@@ -157,7 +168,7 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
     }
     p.kernel = bbo::fit_kernel_for(C, Hs, p.dp);
     if (!p.kernel) return BBO_ERR_UNSUPPORTED;
-    p.per_sm = kernel_occupancy(p.kernel, p.NT, plain);
+    p.per_sm = kernel_occupancy(p.kernel, p.NT, plain, smem_optin);
     if (p.per_sm < 1) continue;
     // Pipelined schedule: where the fit sits alone on its SM anyway and batches span several
     // sub-tiles, two extra warps run the output layer of one sub-tile under the gradient tiles of
@@ -165,7 +176,7 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
     if (TB == 32 && p.per_sm == 1 && Hs >= bbo::kPipeHsMin && maxB > TB && bbo::pipe_extra_warps(Hs) == 2) {
       const void* k = bbo::fit_kernel_for(C, Hs, p.dp, true);
       const size_t sm = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
-      if (k && sm <= budget && kernel_occupancy(k, p.NT + 64, sm) >= 1) {
+      if (k && sm <= budget && kernel_occupancy(k, p.NT + 64, sm, smem_optin) >= 1) {
         p.extra_warps = 2;
         p.NT += 64;
         p.smem = sm;
@@ -195,6 +206,7 @@ struct FitBuffers {  // device scratch of one evaluation
   const int32_t* pi;
   float* trace;
   float* keep_theta;
+  const int32_t* config_keys;  // per-configuration keys of the random streams (null: position + base)
 };
 
 // Orders the fits for launch.  Grids are dispatched in launch order, so the fits are first cut
@@ -275,7 +287,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     bbo::FitArgs a{};
     a.X = Xk; a.y = y; a.pi = buf.pi; a.configs = buf.configs; a.fits = buf.fits + g.begin;
     a.fold_scores = buf.fold_scores; a.trace = buf.trace; a.keep_theta = buf.keep_theta;
-    a.n_fits = g.count; a.n_configs = n_configs; a.config_base = config_base;
+    a.n_fits = g.count; a.n_configs = n_configs; a.config_base = config_base; a.config_keys = buf.config_keys;
     a.solver = solver; a.metric = metric; a.extra_warps = g.plan.extra_warps;
     a.Xt = ho.Xt; a.yt = ho.yt; a.n_test = ho.n_test;
     a.n = n; a.d = d; a.dp = g.plan.dp; a.C = C; a.CS = g.plan.CS; a.K = K; a.task = task;
@@ -284,8 +296,6 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     a.tmem_cols = g.plan.tmem_cols;
     cudaStream_t s = side ? env.aux[gi % env.n_aux] : env.main;
     void* kargs[] = {&a};
-    // groups of different width may share one kernel instance: its limit is per launch
-    if ((e = cudaFuncSetAttribute(g.plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.plan.smem)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
     if ((e = cudaLaunchKernel(g.plan.kernel, dim3(g.count), dim3(g.plan.NT), kargs, g.plan.smem, s)) != cudaSuccess) { *cuda_err = e; return BBO_ERR_CUDA; }
     ++*launches;
   }
@@ -339,8 +349,10 @@ int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out) {
   int dev = o.device;
   if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return BBO_ERR_CUDA;
   if (dev >= count || o.n_classes < 0 || o.n_classes > kMaxClasses || o.trace_steps < 0 || o.config_index_base < 0 ||
-      o.solver < 0 || o.solver > BBO_SOLVER_SGD || o.metric < 0 || o.metric > BBO_METRIC_ALT)
+      o.solver < 0 || o.solver > BBO_SOLVER_SGD || o.metric < 0 || o.metric > BBO_METRIC_ALT ||
+      o.variant < 0 || o.variant > BBO_VARIANT_TF32)
     return BBO_ERR_INVALID_ARG;
+  if (o.variant == BBO_VARIANT_TF32) return BBO_ERR_UNSUPPORTED;  // not built: it cannot meet the score tolerance (see the header)
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return BBO_ERR_CUDA;
   if (prop.major != 10) return BBO_ERR_UNSUPPORTED;  // the kernels are built for sm_100a only
@@ -375,7 +387,7 @@ int bbo_mlp_cv_destroy(bbo_mlp_cv* h) {
   cudaStreamSynchronize(h->stream);
   h->configs.release(); h->fits.release(); h->fold_scores.release(); h->trace.release();
   h->theta.release(); h->xpad.release(); h->xpad_t.release(); h->hx.release(); h->hy.release(); h->hscores.release();
-  h->dbg_f.release(); h->pi.release(); h->misc.release(); h->dbg_i.release(); h->dbg_u.release();
+  h->dbg_f.release(); h->pi.release(); h->misc.release(); h->dbg_i.release(); h->dbg_u.release(); h->keys.release();
   if (h->ev0) cudaEventDestroy(h->ev0);
   if (h->ev1) cudaEventDestroy(h->ev1);
   if (h->evf0) cudaEventDestroy(h->evf0);
@@ -394,7 +406,8 @@ int bbo_mlp_cv_destroy(bbo_mlp_cv* h) {
 // (Xt, yt) are scored.
 static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64, int32_t d, int32_t task,
                      int32_t K, const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed,
-                     float* out_scores, const float* Xt, const float* yt, int64_t n_test64) {
+                     float* out_scores, const float* Xt, const float* yt, int64_t n_test64,
+                     const int32_t* config_keys = nullptr) {
   if (!h || !X || !y || !configs || !out_scores) return BBO_ERR_INVALID_ARG;
   const bool holdout = Xt != nullptr;
   if (n64 < 2 || d < 1 || n_configs < 1) return BBO_ERR_INVALID_ARG;
@@ -406,6 +419,17 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
   int maxH, maxB;
   int rc = check_configs(configs, n_configs, &maxH, &maxB);
   if (rc != BBO_OK) return rc;
+  if (config_keys)
+    for (int c = 0; c < n_configs; ++c)
+      if (config_keys[c] < 0 || config_keys[c] >= (1 << 28)) return BBO_ERR_INVALID_ARG;
+  // shape against the kernel caps before anything is reserved or enqueued (class count at its largest)
+  if (d > kMaxFeatures || maxH > kMaxHidden) return BBO_ERR_UNSUPPORTED;
+  {
+    Plan probe;
+    const int Cmax = task == BBO_TASK_REGRESSION ? 1 : (h->opt.n_classes > 0 ? h->opt.n_classes : 2);
+    rc = plan_bucket(h->smem_optin, (int)n64, d, Cmax, K, bbo::round_up(maxH, 8), maxB, h->opt.trace_steps > 0, true, &probe);
+    if (rc != BBO_OK) return rc;
+  }
   DeviceGuard g(h->device);
   if (!is_device_ptr(X, h->device) || !is_device_ptr(y, h->device) || !is_device_ptr(out_scores, h->device))
     return BBO_ERR_INVALID_ARG;
@@ -449,6 +473,12 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
   BBO_CUDA(h, h->fits.reserve(n_fits));
   BBO_CUDA(h, h->fold_scores.reserve(n_fits));
   BBO_CUDA(h, h->pi.reserve(n));
+  const int32_t* dkeys = nullptr;
+  if (config_keys) {
+    BBO_CUDA(h, h->keys.reserve(n_configs));
+    BBO_CUDA(h, cudaMemcpyAsync(h->keys.p, config_keys, sizeof(int32_t) * (size_t)n_configs, cudaMemcpyHostToDevice, s));
+    dkeys = h->keys.p;
+  }
   float* trace = nullptr;
   if (tracing) {
     const size_t cnt = (size_t)n_fits * h->opt.trace_steps;
@@ -493,7 +523,7 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
   LaunchEnv env;
   env.smem_optin = h->smem_optin; env.main = s; env.aux = h->aux; env.n_aux = kAuxStreams;
   env.fork = h->fork; env.join = h->join;
-  FitBuffers buf{h->configs.p, h->fits.p, h->fold_scores.p, h->pi.p, trace, keep};
+  FitBuffers buf{h->configs.p, h->fits.p, h->fold_scores.p, h->pi.p, trace, keep, dkeys};
   BBO_CUDA(h, cudaEventRecord(h->evf0, s));
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, h->opt.trace_steps, maxB,
@@ -518,6 +548,13 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
 int bbo_mlp_cv_eval(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d, int32_t task, int32_t K,
                     const bbo_mlp_config* configs, int32_t n_configs, uint64_t seed, float* out_scores) {
   return eval_impl(h, X, y, n, d, task, K, configs, n_configs, seed, out_scores, nullptr, nullptr, 0);
+}
+
+int bbo_mlp_cv_eval_keyed(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, int32_t d, int32_t task, int32_t K,
+                          const bbo_mlp_config* configs, const int32_t* config_keys, int32_t n_configs, uint64_t seed,
+                          float* out_scores) {
+  if (!config_keys) return BBO_ERR_INVALID_ARG;
+  return eval_impl(h, X, y, n, d, task, K, configs, n_configs, seed, out_scores, nullptr, nullptr, 0, config_keys);
 }
 
 int bbo_mlp_cv_eval_holdout(bbo_mlp_cv* h, const float* X, const float* y, int64_t n, const float* Xtest,
@@ -719,6 +756,12 @@ struct StaticDevice {
 constexpr int kMaxDevices = 64;
 StaticDevice g_static_dev[kMaxDevices];
 std::mutex g_static_mutex;
+thread_local std::string g_static_error;  // text of the last CUDA error of bbo_mlp_cv_eval_static on this thread
+
+int static_fail(cudaError_t e, const char* what) {
+  g_static_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return e == cudaErrorMemoryAllocation ? BBO_ERR_OOM : BBO_ERR_CUDA;
+}
 
 // One-off set-up for the current device: device address of the scratch array and the
 // device limits the launch plan needs.
@@ -749,6 +792,7 @@ int static_device_setup(int dev, StaticDevice* out) {
 extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float* y, int64_t n64, int32_t d,
                                       int32_t task, int32_t K, int32_t n_classes, const bbo_mlp_config* configs,
                                       int32_t n_configs, uint64_t seed, float* out_scores) {
+  g_static_error.clear();
   if (!X || !y || !configs || !out_scores) return BBO_ERR_INVALID_ARG;
   if (n64 < 2 || d < 1 || K < 2 || K > n64 || n_configs < 1 || n_classes < 0 || n_classes > kMaxClasses)
     return BBO_ERR_INVALID_ARG;
@@ -812,13 +856,18 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
   LaunchEnv env;  // no side streams: creating them would be a resource allocation
   env.smem_optin = sd.smem_optin;
   env.main = s;
-  FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr};
+  FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr, nullptr};
   int launches = 0;
   cudaError_t cuda_err = cudaSuccess;
   rc = launch_all_fits(env, buf, Xk, y, n, d, C, K, task, configs, n_configs, seed, 0, maxB, 0, BBO_SOLVER_ADAM,
                        BBO_METRIC_DEFAULT, HoldoutRows{}, &launches, &cuda_err);
+  if (rc == BBO_ERR_CUDA) return static_fail(cuda_err, "launch_all_fits");
   if (rc != BBO_OK) return rc;
   bbo::fold_mean_kernel<<<(n_configs + 127) / 128, 128, 0, s>>>(fold_scores, n_configs, K, out_scores);
-  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return BBO_ERR_CUDA;
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return static_fail(e, "fold mean / stream synchronisation");
   return BBO_OK;
 }
+
+extern "C" const char* bbo_mlp_cv_static_last_cuda_error(void) { return g_static_error.c_str(); }

@@ -28,6 +28,7 @@ struct FitArgs {
   float* keep_theta;     // parameters of fit (n_configs-1, K-1) in dense layout, or null
   int32_t n_fits, n_configs;
   int32_t config_base;   // added to a configuration's list index when keying its random streams
+  const int32_t* config_keys;  // [n_configs] keys of the random streams, replacing index + base (null: unused)
   int32_t n, d, dp, C, CS, K, task;
   int32_t Hs;            // padded hidden width shared by every fit of this launch
   int32_t TB;            // rows per sub-tile (multiple of 4, at most 32)

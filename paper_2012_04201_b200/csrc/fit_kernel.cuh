@@ -361,7 +361,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
   const int2 cf = a.fits[q];
   const int config = cf.x, fold = cf.y;
-  const uint32_t rng_config = (uint32_t)(config + a.config_base);  // index that keys the random streams
+  const uint32_t rng_config = a.config_keys ? (uint32_t)a.config_keys[config] : (uint32_t)(config + a.config_base);  // keys the random streams
   const Config c = a.configs[config];
   const int H = c.hidden, d = a.d, CS = a.CS, TB = a.TB;
   const int dp = DPC ? DPC : a.dp;

@@ -231,6 +231,16 @@ def test_error_codes(binding):
     with pytest.raises(binding.BboError) as e:
         h.eval(X, y, 0, 5, big, 0)
     assert e.value.code == binding.BBO_ERR_UNSUPPORTED
+    # a shape over the caps is turned away before any scratch is reserved for it
+    free0 = torch.cuda.mem_get_info()[0]
+    wide = torch.zeros(16, 100000, device="cuda")
+    yw = torch.zeros(16, device="cuda")
+    free1 = torch.cuda.mem_get_info()[0]
+    with pytest.raises(binding.BboError) as e:
+        h.eval(wide, yw, 1, 2, wl["configs"], 0)
+    assert e.value.code == binding.BBO_ERR_UNSUPPORTED
+    assert torch.cuda.mem_get_info()[0] == free1
+    del wide, yw, free0
     out = torch.empty(8, device="cuda")
     rc = binding.bbo_mlp_cv_eval(h._h, wl["X"].ctypes.data, y.data_ptr(), 150, 4, 0, 5, wl["configs"], 0, out.data_ptr())
     assert rc == binding.BBO_ERR_INVALID_ARG           # host pointer where a device pointer is required
@@ -255,6 +265,40 @@ def test_split_list_with_index_base_equals_unsplit_call(binding):
         parts.append(h.eval(X, y, wl["task"], 5, wl["configs"][b:e], wl["seed"]).cpu().numpy())
         h.close()
     assert np.array_equal(np.concatenate(parts), whole["scores"])
+
+
+def test_cost_balanced_split_with_keys_equals_unsplit_call(binding):
+    """One list dealt to three handles by estimated cost, every entry keyed by its position in
+    the unsplit list (the multi-GPU path of bench.py, here on one GPU)."""
+    from paper_2012_04201_b200 import sharding
+    wl = W.workload("digits2048", n_configs=13, epochs=3)
+    whole = gpu_eval(binding, wl, wl["configs"])
+    X = torch.from_numpy(wl["X"]).cuda()
+    y = torch.from_numpy(wl["y"]).cuda()
+    assign = sharding.balanced_assignment(sharding.config_costs(wl["configs"], 1797, 64, 10, 5), 3)
+    full = np.full(13, np.nan, np.float32)
+    for rank in range(3):
+        mine = sharding.shard_indices(assign, rank)
+        h = binding.MlpCv(config_index_base=1000)   # ignored by the keyed call
+        full[mine] = h.eval(X, y, wl["task"], 5, wl["configs"][mine], wl["seed"], config_keys=mine).cpu().numpy()
+        h.close()
+    assert np.array_equal(full, whole["scores"])
+    h = binding.MlpCv()
+    with pytest.raises(binding.BboError) as e:
+        h.eval(X, y, wl["task"], 5, wl["configs"][:2], wl["seed"], config_keys=np.array([0, -1], np.int32))
+    assert e.value.code == binding.BBO_ERR_INVALID_ARG
+    h.close()
+
+
+def test_variant_option(binding):
+    h = binding.MlpCv(variant=binding.VARIANT_FP32)
+    h.close()
+    with pytest.raises(binding.BboError) as e:
+        binding.MlpCv(variant=binding.VARIANT_TF32)      # named in the header, not built
+    assert e.value.code == binding.BBO_ERR_UNSUPPORTED
+    with pytest.raises(binding.BboError) as e:
+        binding.MlpCv(variant=7)
+    assert e.value.code == binding.BBO_ERR_INVALID_ARG
 
 
 def test_register_fma_rate_is_near_the_nominal_peak(binding):

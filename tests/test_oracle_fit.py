@@ -63,6 +63,58 @@ def test_step_count_and_short_last_batch():
     assert np.isfinite(r["trace"][0, :6]).all() and np.isnan(r["trace"][0, 6:]).all()
 
 
+def test_minibatch_fit_replayed_step_by_step():
+    # A fit with several minibatches per epoch and a short last batch (120 training rows, B = 50:
+    # 50, 50, 20), replayed outside the fit loop from its parts: the epoch order export, the
+    # minibatch loss/gradient export and the Adam export (double mode, so that the comparison is
+    # not about rounding).  Pins the slicing rows = order[s B : (s+1) B], the per-batch mean over
+    # the true batch size, the step counter running across epochs and the reshuffle per epoch.
+    wl = W.workload("iris8")
+    X, y = wl["X"].astype(np.float64), wl["y"].astype(np.float64)
+    cfg = one_config(hidden=6, batch_size=50, epochs=2, alpha=0.3, lr=0.02, beta1=0.8, beta2=0.95, eps=1e-7)
+    config, fold, seed = 0, 3, 11
+    r = oracle.cv_fits(wl["X"], wl["y"], 0, 5, cfg, seed, [config], [fold], mode=1, trace_steps=8, want_theta=True)
+    th0 = oracle.init_params(4, 6, 3, seed, config, fold)
+    hp = [float(np.float32(v)) for v in (0.02, 0.8, 0.95, 1e-7)]
+    grads, losses = [], []
+    for e in range(2):
+        order = oracle.epoch_order(150, 5, seed, config, fold, e)
+        assert len(order) == 120
+        for s in range(3):
+            rows = order[s * 50:(s + 1) * 50]
+            assert len(rows) == (50, 50, 20)[s]
+            th = th0 if not grads else oracle.adam_steps(1, th0, np.zeros_like(th0), np.zeros_like(th0), np.array(grads), *hp)[0]
+            loss, g = oracle.loss_grad(1, 4, 6, 3, 0, float(np.float32(0.3)), th, X[rows], y[rows])
+            grads.append(g); losses.append(loss)
+    th_final = oracle.adam_steps(1, th0, np.zeros_like(th0), np.zeros_like(th0), np.array(grads), *hp)[0]
+    np.testing.assert_allclose(r["trace"][0, :6], losses, rtol=1e-12)
+    assert np.all(np.isnan(r["trace"][0, 6:]))
+    np.testing.assert_allclose(r["theta"], th_final, rtol=1e-11, atol=1e-13)
+    # a wrong slice (e.g. dropping the short batch, or reusing epoch 0's order) would not reproduce it
+    assert not np.array_equal(oracle.epoch_order(150, 5, seed, config, fold, 0), oracle.epoch_order(150, 5, seed, config, fold, 1))
+
+
+def test_diverged_fits_nan_maps_to_minus_infinity_and_class_zero():
+    # A learning rate of 1e20 turns the parameters into NaN within a few steps.  Regression: the
+    # held-out error is NaN and the score is -inf (never NaN).  Classification: every logit is NaN,
+    # NaN never wins the ascending strict-> scan, so the prediction is class 0 (the lowest index,
+    # which is also what a tie between equal logits gives) and the accuracy is the share of
+    # class-0 rows in the held-out fold.
+    wl = W.workload("diabetes4096", n_configs=1)
+    cfg = one_config(hidden=6, epochs=40, lr=1e20, batch_size=64)
+    r = oracle.cv_fits(wl["X"], wl["y"], 1, 5, cfg, 0, [0, 0], [0, 1], want_theta=True)
+    assert np.isnan(r["theta"]).any()
+    assert np.all(np.isneginf(r["scores"]))
+    ev = oracle.cv_eval(wl["X"], wl["y"], 1, 5, cfg, 0)
+    assert np.isneginf(ev["scores"][0]) and not np.isnan(ev["fold_scores"]).any()
+    wl = W.workload("iris8")
+    _, fo = oracle.fold_split(150, 5, 0)
+    r = oracle.cv_fits(wl["X"], wl["y"], 0, 5, cfg, 0, [0, 0], [0, 1], want_theta=True)
+    assert np.isnan(r["theta"]).any()
+    for f, score in zip((0, 1), r["scores"]):
+        assert abs(score - np.mean(wl["y"][fo == f] == 0)) < 1e-6
+
+
 def test_float_and_double_traces_agree_over_50_steps():
     wl = W.workload("breast128", n_configs=6)
     a = oracle.cv_eval(wl["X"], wl["y"], 0, 5, wl["configs"], 0, mode=0, trace_steps=50)

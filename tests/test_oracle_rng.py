@@ -144,6 +144,19 @@ def test_glorot_init_bounds_and_moments():
     w = philox_int([0, 7, 3, (2 << 28) | 0], [0, 0])
     u = np.float32(w[1] >> 8) * np.float32(2.0**-24)
     assert th[1] == float(b1 * (np.float32(2.0) * u - np.float32(1.0)))
+
+    # one hand-recomputed element of every other block of the parameter vector: the layer tag
+    # (1 = b1, 2 = W2, 3 = b2) sits in the low bits of the last counter word, element i is word
+    # i & 3 of block i >> 2, W2 is indexed j * C + o, and each layer uses its own bound
+    def draw(layer, idx, bound):
+        w = philox_int([idx >> 2, 7, 3, (2 << 28) | layer], [0, 0])[idx & 3]
+        return float(bound * (np.float32(2.0) * (np.float32(w >> 8) * np.float32(2.0**-24)) - np.float32(1.0)))
+
+    assert th[d * H + 5] == draw(1, 5, b1)                                   # b1[5]
+    assert th[d * H + H + 37 * C + 4] == draw(2, 37 * C + 4, b2)             # W2[37][4]
+    assert th[d * H + H + H * C + 9] == draw(3, 9, b2)                       # b2[9]
+    assert th[3 * H + 130] == draw(0, 3 * H + 130, b1)                       # W1[3][130]
+    assert len({draw(t, 9, b2) for t in (1, 2, 3)}) == 3                     # swapping two tags would show
     # different (config, fold) -> different draw; all values float32-representable
     assert not np.array_equal(th, oracle.init_params(d, H, C, 0, 7, 4))
     assert np.array_equal(th, th.astype(np.float32).astype(np.float64))

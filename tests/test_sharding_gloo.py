@@ -28,6 +28,25 @@ def test_shard_bounds_cover_the_list():
         sharding.shard_bounds(4, 2, 2)
 
 
+def test_cost_balanced_deal_is_a_partition_and_balanced():
+    wl = W.workload("digits2048", n_configs=400)
+    cfg = wl["configs"]
+    costs = sharding.config_costs(cfg, 1797, 64, 10, 5)
+    assert costs.shape == (400,) and np.all(costs > 0)
+    # costlier by construction: more epochs, wider, smaller batches
+    more = cfg.copy(); more["epochs"] *= 2
+    assert np.all(sharding.config_costs(more, 1797, 64, 10, 5) > costs)
+    for world in (1, 2, 3, 8):
+        a = sharding.balanced_assignment(costs, world)
+        parts = [sharding.shard_indices(a, r) for r in range(world)]
+        assert sorted(np.concatenate(parts).tolist()) == list(range(400))     # every entry exactly once
+        load = np.array([costs[p].sum() for p in parts])
+        assert load.max() / load.mean() < 1.10                                 # within 10 % of even
+        assert np.array_equal(a, sharding.balanced_assignment(costs, world))   # deterministic
+    with pytest.raises(ValueError):
+        sharding.balanced_assignment(costs, 0)
+
+
 def _free_port():
     s = socket.socket()
     s.bind(("127.0.0.1", 0))
@@ -61,6 +80,47 @@ def _rank_main(rank, world, port, out_path):
         np.save(out_path, np.concatenate([full.numpy(), t.numpy()]))
     dist.barrier()
     dist.destroy_process_group()
+
+
+def _balanced_rank_main(rank, world, port, out_path):
+    import oracle
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = W.workload("iris8", n_configs=11, epochs=3)
+    cfg, K = wl["configs"], wl["n_folds"]
+    costs = sharding.config_costs(cfg, wl["X"].shape[0], wl["X"].shape[1], 3, K)
+    assign = sharding.balanced_assignment(costs, world)
+    mine = sharding.shard_indices(assign, rank)
+    fc = np.repeat(mine, K)
+    ff = np.tile(np.arange(K), mine.size)
+    # the checker keys the random streams by position in the list it is given: passing the whole
+    # list and the positions of this rank's entries is what bbo_mlp_cv_eval_keyed does on the device
+    fits = oracle.cv_fits(wl["X"], wl["y"], wl["task"], K, cfg, wl["seed"], fc, ff, n_threads=1)["scores"]
+    local = np.zeros(mine.size, np.float32)
+    for i in range(mine.size):
+        acc = np.float32(0)
+        for f in range(K):
+            acc = np.float32(acc + np.float32(fits[i * K + f]))
+        local[i] = acc / np.float32(K)
+    full = sharding.gather_scores_by_assignment(local, assign, rank, world, dist)
+    if rank == 0:
+        np.save(out_path, full.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_cost_balanced_ranks_reproduce_the_unsplit_scores(tmp_path, world):
+    import oracle
+
+    out = str(tmp_path / "gathered.npy")
+    mp.spawn(_balanced_rank_main, args=(world, _free_port(), out), nprocs=world, join=True)
+    got = np.load(out)
+    wl = W.workload("iris8", n_configs=11, epochs=3)
+    ref = oracle.cv_eval(wl["X"], wl["y"], wl["task"], wl["n_folds"], wl["configs"], wl["seed"])["scores"]
+    assert np.array_equal(got.astype(np.float64), ref)
 
 
 def test_two_ranks_reproduce_the_unsplit_scores(tmp_path):
