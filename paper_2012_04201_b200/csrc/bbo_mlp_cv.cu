@@ -25,6 +25,13 @@ constexpr int kAuxStreams = 32;  // buckets of different hidden width overlap on
 constexpr int kMaxRows = 16384;  // fold permutation sorts in one CTA's shared memory
 constexpr int kMaxFeatures = 16384, kMaxHidden = 8192;  // beyond any shape shared memory admits; keeps the size arithmetic in int
 
+// Device limits the launch plan needs.
+struct DeviceLimits {
+  int smem_optin = 0;   // largest shared memory of one CTA (static + dynamic)
+  int smem_per_sm = 0;  // shared memory of one SM
+  int regs_per_sm = 0;  // 32-bit registers of one SM
+};
+
 template <typename T>
 struct DevBuf {
   T* p = nullptr;
@@ -52,7 +59,7 @@ struct bbo_mlp_cv {
   cudaStream_t stream = nullptr;
   bbo_mlp_cv_options opt{};
   int sm_count = 0;
-  int smem_optin = 0;
+  DeviceLimits lim;
   std::string cuda_error;
   // scratch
   DevBuf<bbo::Config> configs;
@@ -112,36 +119,43 @@ struct Plan {
   const void* kernel;
 };
 
-// Resident CTAs per SM of a fit kernel instance (0 if it cannot launch).  The dynamic
-// shared-memory limit of an instance is always set to the device's opt-in maximum, never to the
-// size of one launch: the attribute is global to the process, and handles on different threads
-// share the instances.
-int kernel_occupancy(const void* kernel, int threads, size_t smem, int smem_optin) {
+// Resident CTAs per SM of a fit kernel instance (0 if it cannot launch), from the kernel's own
+// registers and static shared memory, the launch's dynamic shared memory and threads, and the
+// tensor-memory columns each CTA allocates (512 per SM; the occupancy query of the runtime
+// does not know about those).  Also raises the instance's dynamic shared-memory limit to the
+// device's opt-in maximum -- always that value, never the size of one launch: the attribute is
+// global to the process, and handles on different threads share the instances.
+int kernel_occupancy(const void* kernel, int threads, size_t smem, int tmem_cols, const DeviceLimits& lim) {
   cudaFuncAttributes attr;
   if (cudaFuncGetAttributes(&attr, kernel) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
-  const int max_dynamic = smem_optin - (int)attr.sharedSizeBytes;  // the opt-in limit covers static + dynamic
+  const int max_dynamic = lim.smem_optin - (int)attr.sharedSizeBytes;  // the opt-in limit covers static + dynamic
   if ((size_t)max_dynamic < smem ||
       cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dynamic) != cudaSuccess ||
       cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
-  int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem) != cudaSuccess) {
-    cudaGetLastError();
-    return 0;
-  }
-  return per_sm;
+  if (threads > attr.maxThreadsPerBlock) return 0;
+  const int warps = (threads + 31) / 32;
+  const int regs_per_warp = bbo::round_up(attr.numRegs, 8) * 32;
+  const int by_smem = (int)((size_t)lim.smem_per_sm / (smem + attr.sharedSizeBytes + 1024));  // 1 KB per CTA is reserved
+  int by_regs = lim.regs_per_sm / (regs_per_warp * warps);
+  // the registers sit in four partitions of a quarter each; warps are dealt to the partitions in turn
+  while (by_regs > 1 && (by_regs * warps + 3) / 4 * regs_per_warp > lim.regs_per_sm / 4) --by_regs;
+  const int by_tmem = tmem_cols > 0 ? 512 / tmem_cols : 32;
+  const int by_threads = 2048 / threads;
+  return std::max(0, std::min(std::min(by_smem, by_regs), std::min(std::min(by_tmem, by_threads), 32)));
 }
 
 // Plans the launch of fits of padded width Hs.  Threads: one per gradient tile of W1 (8 rows x
 // 8 columns) and one per hidden unit.  Sub-tile height: the largest of 32, 16, 8 that fits.
 // probe_only: skip the occupancy queries (no CUDA calls), used by the caps query.
-int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bool tracing, bool probe_only,
+int plan_bucket(const DeviceLimits& lim, int n, int d, int C, int K, int Hs, int maxB, bool tracing, bool probe_only,
                 Plan* out) {
+  const int smem_optin = lim.smem_optin;
   Plan p{};
   p.C = C;
   p.CS = bbo::round_up(C, 4);
@@ -168,7 +182,7 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
     }
     p.kernel = bbo::fit_kernel_for(C, Hs, p.dp);
     if (!p.kernel) return BBO_ERR_UNSUPPORTED;
-    p.per_sm = kernel_occupancy(p.kernel, p.NT, plain, smem_optin);
+    p.per_sm = kernel_occupancy(p.kernel, p.NT, plain, p.tmem_cols, lim);
     if (p.per_sm < 1) continue;
     // Pipelined schedule: where the fit sits alone on its SM anyway and batches span several
     // sub-tiles, two extra warps run the output layer of one sub-tile under the gradient tiles of
@@ -176,7 +190,7 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
     if (TB == 32 && p.per_sm == 1 && Hs >= bbo::kPipeHsMin && maxB > TB && bbo::pipe_extra_warps(Hs) == 2) {
       const void* k = bbo::fit_kernel_for(C, Hs, p.dp, true);
       const size_t sm = bbo::fit_smem_bytes(d, p.dp, Hs, C, p.CS, TB, p.order_bytes, p.loss_cap, p.n_sort, true);
-      if (k && sm <= budget && kernel_occupancy(k, p.NT + 64, sm, smem_optin) >= 1) {
+      if (k && sm <= budget && kernel_occupancy(k, p.NT + 64, sm, p.tmem_cols, lim) >= 1) {
         p.extra_warps = 2;
         p.NT += 64;
         p.smem = sm;
@@ -191,7 +205,7 @@ int plan_bucket(int smem_optin, int n, int d, int C, int K, int Hs, int maxB, bo
 
 // Where the fits of one evaluation run: the caller's stream plus optional side streams.
 struct LaunchEnv {
-  int smem_optin = 0;
+  DeviceLimits lim;
   cudaStream_t main = nullptr;
   cudaStream_t* aux = nullptr;  // may be null: everything runs on `main`
   int n_aux = 0;
@@ -265,7 +279,7 @@ int launch_all_fits(const LaunchEnv& env, const FitBuffers& buf, const float* Xk
     int j = i;
     while (j < n_fits && items[j].Hs == items[i].Hs && items[j].tier == items[i].tier) ++j;
     Group g{i, j - i, {}};
-    const int rc = plan_bucket(env.smem_optin, n, d, C, K, items[i].Hs, maxB, trace_steps > 0, false, &g.plan);
+    const int rc = plan_bucket(env.lim, n, d, C, K, items[i].Hs, maxB, trace_steps > 0, false, &g.plan);
     if (rc != BBO_OK) return rc;
     groups.push_back(g);
     i = j;
@@ -362,7 +376,9 @@ int bbo_mlp_cv_create(const bbo_mlp_cv_options* opt, bbo_mlp_cv** out) {
   h->stream = static_cast<cudaStream_t>(o.stream);
   h->opt = o;
   h->sm_count = prop.multiProcessorCount;
-  h->smem_optin = (int)prop.sharedMemPerBlockOptin;
+  h->lim.smem_optin = (int)prop.sharedMemPerBlockOptin;
+  h->lim.smem_per_sm = (int)prop.sharedMemPerMultiprocessor;
+  h->lim.regs_per_sm = prop.regsPerMultiprocessor;
   DeviceGuard g(dev);
   if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess ||
       cudaEventCreate(&h->evf0) != cudaSuccess || cudaEventCreate(&h->evf1) != cudaSuccess) {
@@ -427,7 +443,7 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
   {
     Plan probe;
     const int Cmax = task == BBO_TASK_REGRESSION ? 1 : (h->opt.n_classes > 0 ? h->opt.n_classes : 2);
-    rc = plan_bucket(h->smem_optin, (int)n64, d, Cmax, K, bbo::round_up(maxH, 8), maxB, h->opt.trace_steps > 0, true, &probe);
+    rc = plan_bucket(h->lim, (int)n64, d, Cmax, K, bbo::round_up(maxH, 8), maxB, h->opt.trace_steps > 0, true, &probe);
     if (rc != BBO_OK) return rc;
   }
   DeviceGuard g(h->device);
@@ -521,7 +537,7 @@ static int eval_impl(bbo_mlp_cv* h, const float* X, const float* y, int64_t n64,
   ++launches;
 
   LaunchEnv env;
-  env.smem_optin = h->smem_optin; env.main = s; env.aux = h->aux; env.n_aux = kAuxStreams;
+  env.lim = h->lim; env.main = s; env.aux = h->aux; env.n_aux = kAuxStreams;
   env.fork = h->fork; env.join = h->join;
   FitBuffers buf{h->configs.p, h->fits.p, h->fold_scores.p, h->pi.p, trace, keep, dkeys};
   BBO_CUDA(h, cudaEventRecord(h->evf0, s));
@@ -692,7 +708,7 @@ int bbo_mlp_cv_query_caps(bbo_mlp_cv* h, int32_t d, int32_t n_classes, int32_t* 
   // widest hidden layer for (d, C) on a 1797-row, 5-fold problem with the smallest sub-tile
   auto fits_H = [&](int dd, int H) {
     Plan p;
-    return plan_bucket(h->smem_optin, 1797, dd, n_classes, 5, bbo::round_up(H, 8), 1, false, true, &p) == BBO_OK;
+    return plan_bucket(h->lim, 1797, dd, n_classes, 5, bbo::round_up(H, 8), 1, false, true, &p) == BBO_OK;
   };
   if (max_hidden) {
     int lo = 0, hi = 4096;
@@ -751,7 +767,8 @@ namespace {
 struct StaticDevice {
   bool ready = false;
   unsigned char* base = nullptr;
-  int sm_count = 0, smem_optin = 0, major = 0;
+  int sm_count = 0, major = 0;
+  DeviceLimits lim;
 };
 constexpr int kMaxDevices = 64;
 StaticDevice g_static_dev[kMaxDevices];
@@ -775,7 +792,9 @@ int static_device_setup(int dev, StaticDevice* out) {
       return BBO_ERR_CUDA;
     }
     if (cudaDeviceGetAttribute(&sd.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sd.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sd.lim.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sd.lim.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sd.lim.regs_per_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sd.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
       cudaGetLastError();
       return BBO_ERR_CUDA;
@@ -854,7 +873,7 @@ extern "C" int bbo_mlp_cv_eval_static(void* stream, const float* X, const float*
   }
   if (launch_fold_permutation(n, seed, pi, s) != cudaSuccess) return BBO_ERR_CUDA;
   LaunchEnv env;  // no side streams: creating them would be a resource allocation
-  env.smem_optin = sd.smem_optin;
+  env.lim = sd.lim;
   env.main = s;
   FitBuffers buf{dcfg, dfits, fold_scores, pi, nullptr, nullptr, nullptr};
   int launches = 0;

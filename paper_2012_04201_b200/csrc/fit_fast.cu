@@ -12,7 +12,7 @@ namespace bbo {
 template <>
 const void* fast_fit_kernel<BBO_HSC>(bool pipe) {
   constexpr int NT = fast_threads(BBO_HSC);
-#if BBO_HSC >= 128
+#if BBO_HSC >= 184
   constexpr int NTP = NT + 64 <= kMaxFitThreads ? NT + 64 : NT + 32;  // one or two extra warps for the output layer
   if (pipe) return reinterpret_cast<const void*>(&mlp_cv_fit_kernel<kFastClasses, BBO_HSC, kFastDp, NTP, 1, true>);
 #else

@@ -18,14 +18,20 @@ constexpr int kFastDp = 64, kFastClasses = 10, kFastHsMin = 56, kFastHsMax = 200
 
 // Pipelined schedule (gradient tiles of one sub-tile overlap the output layer of the next, run by
 // extra warps): built for the fast-path widths that sit alone on an SM.
-constexpr int kPipeHsMin = 128;
+constexpr int kPipeHsMin = 184;
 inline int pipe_extra_warps(int Hs) { return (Hs + 31) / 32 * 32 + 64 <= kMaxFitThreads ? 2 : 1; }
 
 // Resident CTAs per SM the compile-time-width instances are built for: the launch bound caps
 // their registers at 65,536 / (CTAs x threads), and shared memory admits that many (the row
-// buffers and parameters of a fit of that width, moments of W1 in tensor memory).
+// buffers and parameters of a fit of that width, moments of W1 in tensor memory).  Four fits per
+// SM up to width 64 and two up to 128 keep about 250 registers per thread.  Widths 136..176 (five
+// or six warps) also run two per SM, at 168 registers and a few hundred bytes of spills: a lone
+// CTA is then 40 % slower, but two of them share an SM at a cost of 10 %, which beats one CTA
+// with the pipelined schedule by 8 %.  Three CTAs of widths 72..96 at 168 registers were 12 %
+// slower than two at 250.  Widths from 184 sit alone on their SM (shared memory) and take the
+// pipelined schedule.
 constexpr int fast_threads(int Hs) { return (Hs + 31) / 32 * 32; }
-constexpr int fast_min_blocks(int Hs) { return fast_threads(Hs) <= 64 ? 4 : (fast_threads(Hs) <= 96 ? 3 : (Hs <= 176 ? 2 : 1)); }
+constexpr int fast_min_blocks(int Hs) { return fast_threads(Hs) <= 64 ? 4 : (Hs <= 176 ? 2 : 1); }
 
 template <int CT> const void* generic_fit_kernel();            // run-time strides
 template <int HSC> const void* fast_fit_kernel(bool pipe);     // compile-time strides; pipe: pipelined schedule
