@@ -38,11 +38,13 @@ from paper_2012_04201_b200 import workloads  # noqa: E402
 METRIC = "mlp_adam_cv_fits_per_sec"
 UNIT = "fits/s"
 SM_COUNT_FP32_LANES = 128  # FP32 lanes per SM on sm_100
-# dram__bytes_read.sum + dram__bytes_write.sum of one fit-kernel launch (ncu capture summarised in
-# profiles/mlp_cv_fit_kernel_small_cases_full.md): the dataset, the labels, the configurations
-# and the fit list, read once; the same for every launch size because weights, moments and
-# activations never leave the SM.
-FIT_KERNEL_DRAM_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one fit-kernel launch on the digits-shaped data
+# (ncu capture of a 29-fit launch, summarised in profiles/mlp_cv_fit_kernel_small_cases_full.md):
+# the dataset, the labels, the configurations and the fit list, read once.  It does not grow with
+# the number of fits in the launch, because weights, moments and activations never leave the SM
+# and every later read of X hits the L2; so the figure is not scaled to the bench's launch size.
+# Other workloads have no capture of their own and report null.
+FIT_KERNEL_DRAM_BYTES_PER_LAUNCH = {"digits_sweep": 632832, "digits2048": 632832}
 
 
 def parse_args():
@@ -413,7 +415,7 @@ def main():
     achieved = work["flops"] / fit_s / 1e12
     roofline = {
         "bound": "alu", "kernel": "mlp_cv_fit_kernel", "achieved": achieved, "peak": fp32_peak, "unit": "TFLOP/s",
-        "frac": achieved / fp32_peak, "traffic": FIT_KERNEL_DRAM_BYTES_PER_LAUNCH,
+        "frac": achieved / fp32_peak, "traffic": FIT_KERNEL_DRAM_BYTES_PER_LAUNCH.get(args.workload),
         "peak_source": f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 x {sm_max:.0f} MHz (max SM clock); "
                        f"HBM/bf16 peaks are {peak_kind} and do not bound this kernel",
         "gemm_only_achieved": work["gemm_flops"] / fit_s / 1e12,
