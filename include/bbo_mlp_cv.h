@@ -184,7 +184,8 @@ int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* ou
  * versions inside a safe exponent range and the IEEE routines outside it.  This export
  * compares the two on the device.  mode 0: square root of the `count` float bit patterns
  * starting at `first`; mode 1: m / (sqrt(v) + eps) on `count` pseudo-random operand triples
- * keyed by `seed`; mode 2: softmax quotients exp(-t) / s, t in [0, 90), s in [1, 16], on
+ * keyed by `seed`; mode 3: the same quotient with denormal or tiny m, so that most results
+ * are denormal; mode 2: softmax quotients exp(-t) / s, t in [0, 90), s in [1, 16], on
  * `count` pseudo-random pairs.  host_out4: HOST [4] = number of
  * bit-level disagreements, number of cases taken by the fast path, and (for diagnosis) the
  * operand bits of one disagreement.                                                       */

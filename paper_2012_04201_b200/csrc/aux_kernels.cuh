@@ -69,7 +69,9 @@ __global__ void debug_rng_kernel(uint64_t seed, const uint32_t* ctr, int64_t cou
 // Debug: counts inputs in the safe range for which the branch-free square root / division
 // differ from the IEEE intrinsics.  mode 0: sqrt(v) and sqrt(v) + eps over the bit patterns first .. first+count-1 (denormals included);
 // mode 1: m / (sqrt(v) + eps) over `count` operand triples drawn from Philox words with
-// exponents spread over the whole float range.  out[0] = mismatches, out[1] = cases the fast
+// exponents spread over the whole float range; mode 3: the same quotient with tiny or denormal
+// m over ordinary v and eps, so that most quotients are denormal, exact ties included (a
+// denominator of exactly 2 under an odd multiple of the smallest denormal).  out[0] = mismatches, out[1] = cases the fast
 // path declared safe, out[2..3] = operands of one mismatch.
 __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, uint64_t count, unsigned long long* out) {
   unsigned long long bad = 0, safe_n = 0;
@@ -92,6 +94,23 @@ __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, 
       ++safe_n;
       const float ref = __fdiv_rn(e, s);
       if (__float_as_uint(q) != __float_as_uint(ref)) { ++bad; out[2] = __float_as_uint(e); out[3] = __float_as_uint(s); }
+    } else if (mode == 3) {
+      const uint4 r = philox4x32_10(seed, 9u, (uint32_t)(i >> 32), 0u, 0u, (uint32_t)i);
+      float m = __uint_as_float((r.x & 0x807FFFFFu) | ((r.w % 48u) << 23));  // denormal .. 2^-80, either sign
+      float vv = __uint_as_float((r.y & 0x007FFFFFu) | ((40u + (r.w >> 8) % 90u) << 23));  // 2^-87 .. 2^2
+      if (((r.w >> 20) & 15u) == 0u) vv = __uint_as_float(r.y & 0x007FFFFFu);              // denormal or zero v
+      const float eps_set[4] = {1e-8f, 0x1p-40f, 1e-3f, 0.75f};
+      float eps = eps_set[(r.w >> 24) & 3u];
+      if ((r.w >> 28) == 0u) {  // denominator exactly 2: odd numerators are exact ties
+        vv = 1.5625f; eps = 0.75f;
+        m = __uint_as_float((r.x & 0x80000000u) | (r.x & 0xFFu));
+      }
+      AdamCert cert;
+      const float q = adam_ratio_fast(m, vv, eps, cert);
+      if ((adam_eps_safe(eps) & cert.ok()) == 0u) continue;
+      ++safe_n;
+      const float ref = adam_ratio_ieee(m, vv, eps);
+      if (__float_as_uint(q) != __float_as_uint(ref)) { ++bad; out[2] = __float_as_uint(m); out[3] = __float_as_uint(vv); }
     } else {
       const uint4 r = philox4x32_10(seed, 7u, (uint32_t)(i >> 32), 0u, 0u, (uint32_t)i);
       const float m = __uint_as_float(r.x);

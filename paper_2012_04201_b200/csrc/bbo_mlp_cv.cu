@@ -670,7 +670,7 @@ int bbo_mlp_cv_debug_exp(bbo_mlp_cv* h, const float* x, int64_t count, float* ou
 
 int bbo_mlp_cv_debug_fast_math(bbo_mlp_cv* h, int32_t mode, uint64_t seed, uint64_t first, uint64_t count,
                                uint64_t* host_out4) {
-  if (!h || !host_out4 || count < 1 || (mode < 0 || mode > 2)) return BBO_ERR_INVALID_ARG;
+  if (!h || !host_out4 || count < 1 || (mode < 0 || mode > 3)) return BBO_ERR_INVALID_ARG;
   DeviceGuard g(h->device);
   cudaStream_t s = h->stream;
   BBO_CUDA(h, h->dbg_u.reserve(8));

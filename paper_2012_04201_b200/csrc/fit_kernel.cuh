@@ -78,30 +78,31 @@ __device__ __forceinline__ float f4_get(const float4& v, int i) {
   return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
 }
 
-// A1 = relu(Xs W1 + b1) for the sub-tile; each thread owns 8 rows x 4 columns, k ascending.
-__device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L, const float* xs, int d, int dp,
-                                               int Hs, int nb, int tid, int nt) {
-  const int JG = Hs >> 2, n_tiles = ((nb + 7) >> 3) * JG;
+// A1 = relu(Xs W1 + b1) for the sub-tile; each thread owns R rows x 4 columns, k ascending.
+template <int R>
+__device__ __forceinline__ void forward_tiles(const FitView& v, const Layout& L, const float* xs, int d, int dp,
+                                              int Hs, int nb, int tid, int nt) {
+  const int JG = Hs >> 2, n_tiles = ((nb + R - 1) / R) * JG;
   const int d4 = d >> 2;
   for (int t = tid; t < n_tiles; t += nt) {
     const int bg = t / JG, jg = t - bg * JG;
-    const int b0 = bg << 3, j0 = jg << 2;
+    const int b0 = bg * R, j0 = jg << 2;
     const float4 bias = *reinterpret_cast<const float4*>(v.W + L.ob1 + j0);
-    float acc[8][4];
+    float acc[R][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { acc[i][0] = bias.x; acc[i][1] = bias.y; acc[i][2] = bias.z; acc[i][3] = bias.w; }
+    for (int i = 0; i < R; ++i) { acc[i][0] = bias.x; acc[i][1] = bias.y; acc[i][2] = bias.z; acc[i][3] = bias.w; }
     const float* xrow = xs + b0 * dp;
     const float* wp = v.W + L.oW1 + j0;
 #pragma unroll 2
     for (int k4 = 0; k4 < d4; ++k4) {
-      float4 xv[8];
+      float4 xv[R];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) xv[i] = *reinterpret_cast<const float4*>(xrow + i * dp + 4 * k4);
+      for (int i = 0; i < R; ++i) xv[i] = *reinterpret_cast<const float4*>(xrow + i * dp + 4 * k4);
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
         const float4 w = *reinterpret_cast<const float4*>(wp + (4 * k4 + kk) * Hs);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < R; ++i) {
           const float x = f4_get(xv[i], kk);
           acc[i][0] = __fmaf_rn(x, w.x, acc[i][0]);
           acc[i][1] = __fmaf_rn(x, w.y, acc[i][1]);
@@ -113,7 +114,7 @@ __device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L
     for (int k = d4 << 2; k < d; ++k) {
       const float4 w = *reinterpret_cast<const float4*>(wp + k * Hs);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < R; ++i) {
         const float x = xrow[i * dp + k];
         acc[i][0] = __fmaf_rn(x, w.x, acc[i][0]);
         acc[i][1] = __fmaf_rn(x, w.y, acc[i][1]);
@@ -122,7 +123,7 @@ __device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L
       }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < R; ++i) {
       float4 o;
       o.x = acc[i][0] > 0.f ? acc[i][0] : 0.f;
       o.y = acc[i][1] > 0.f ? acc[i][1] : 0.f;
@@ -131,6 +132,14 @@ __device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L
       *reinterpret_cast<float4*>(v.A1 + (b0 + i) * L.WP + j0) = o;
     }
   }
+}
+
+// Sub-tiles of at most 16 rows (small minibatches, ragged ends) take 4-row tiles so that all
+// threads share the work; full sub-tiles take 8-row tiles (fewer loads per multiply-add).
+__device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L, const float* xs, int d, int dp,
+                                               int Hs, int nb, int tid, int nt) {
+  if (nb <= 16) forward_tiles<4>(v, L, xs, d, dp, Hs, nb, tid, nt);
+  else forward_tiles<8>(v, L, xs, d, dp, Hs, nb, tid, nt);
 }
 
 // Output layer.  A lane owns one row of the sub-tile and one half of the classes: classes

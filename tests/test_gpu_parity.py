@@ -101,6 +101,12 @@ def test_branch_free_sqrt_and_division_equal_ieee(binding):
         assert out[0] == 0, out
         total_safe += int(out[1])
     assert total_safe > 5e7
+    # tiny and denormal first moments over ordinary denominators: denormal quotients, which long
+    # fits with an L2 term produce all the time, must come out of the fast path, and exactly
+    for seed in (4, 5):
+        out = h.debug_fast_math(3, seed=seed, count=2**31)
+        assert out[0] == 0, out
+        assert out[1] > 0.9 * 2**31, out
     # softmax quotients: exponentials of non-positive numbers over denominators in [1, 16]
     out = h.debug_fast_math(2, seed=3, count=2**30)
     assert out[0] == 0 and out[1] > 1.0e9, out
