@@ -78,7 +78,7 @@ __global__ void debug_fast_math_kernel(int mode, uint64_t seed, uint64_t first, 
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < count; i += (uint64_t)gridDim.x * blockDim.x) {
     if (mode == 0) {
       const float x = __uint_as_float((uint32_t)(first + i));
-      if (!(x < 0x1p+30f)) continue;
+      if (!(x < 0x1p+32f)) continue;
       ++safe_n;
       const float eps = 0x1p-30f;
       const float a = adam_denominator_fast(x, eps), b = __fadd_rn(__fsqrt_rn(x), eps);

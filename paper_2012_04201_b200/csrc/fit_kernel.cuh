@@ -204,14 +204,6 @@ __device__ __forceinline__ void output_logits(const FitView& v, const Layout& L,
   }
 }
 
-// Adam on one parameter with its gradient (L2 term already added for weights).
-__device__ __forceinline__ void adam_one(float& th, float& m, float& vv, float g, float beta1, float beta2,
-                                         float omb1, float omb2, float step, float eps) {
-  m = __fmaf_rn(beta1, m, __fmul_rn(omb1, g));
-  vv = __fmaf_rn(beta2, vv, __fmul_rn(__fmul_rn(omb2, g), g));
-  th = __fsub_rn(th, __fmul_rn(step, adam_ratio_ieee(m, vv, eps)));
-}
-
 // Adam on N parameters held in registers, first pass: moments updated in place, parameters
 // updated with the branch-free ratio.  Returns 1 when every ratio was computed inside the range
 // in which it equals the IEEE result; otherwise the caller discards th[] and redoes the
@@ -782,7 +774,14 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           sgd_group<1>(w1, m1, g1b, c.lr, beta1);
           v.W[off] = w1[0]; v.M[off] = m1[0];
         } else {
-          adam_one(v.W[off], v.M[off], v.V[off], gb2, beta1, beta2, omb1, omb2, step, eps);
+          float w1[1] = {v.W[off]}, m1[1] = {v.M[off]}, v1[1] = {v.V[off]};
+          const float g1b[1] = {gb2};
+          const float wold = w1[0];
+          if (!adam_group_fast<1>(w1, m1, v1, g1b, beta1, beta2, omb1, omb2, step, eps, eps_safe)) {
+            w1[0] = wold;
+            adam_params_ieee<1>(w1, m1, v1, step, eps);
+          }
+          v.W[off] = w1[0]; v.M[off] = m1[0]; v.V[off] = v1[0];
         }
       }
       ++step_no;

@@ -1,7 +1,6 @@
 // Thin wrappers over the sm_100a instructions the fit kernel uses besides plain arithmetic:
-// shared-memory barriers (mbarrier) with bounded waits, bulk asynchronous row copies that
-// complete on such a barrier, and tensor memory (TMEM) used as per-thread scratch through
-// tcgen05.st / tcgen05.ld.  Nothing here multicasts and nothing reads another GPU's memory.
+// tensor memory (TMEM) used as per-thread scratch through tcgen05.alloc / st / ld / dealloc.
+// No tensor-core instruction is issued, nothing multicasts, nothing reads another GPU's memory.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -9,43 +8,6 @@
 namespace bbo {
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// ---- mbarrier ----
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
-}
-__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-// One arrival that also announces `bytes` of asynchronous copies still to land on the barrier.
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-// True once the phase of the given parity has completed.  A pending phase makes the instruction
-// wait for a short, implementation-defined time before it returns false, so a polling loop does
-// not flood the issue slots.
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t done;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(done)
-      : "r"(smem_addr(bar)), "r"(parity)
-      : "memory");
-  return done != 0;
-}
-
-// ---- bulk asynchronous copy global -> shared, completing `bytes` on `bar` ----
-// dst, src 16-byte aligned; bytes a multiple of 16.  No multicast.
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst)),
-               "l"(src), "r"(bytes), "r"(smem_addr(bar))
-               : "memory");
-}
-
-// Orders this thread's earlier shared-memory accesses through ordinary loads and stores before
-// later accesses of the asynchronous copy engine to the same locations.
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---- tensor memory as scratch ----
 // A warp reaches the 32 TMEM lanes 32 * (warp index % 4) ..; with the 32x32b shape thread i of
