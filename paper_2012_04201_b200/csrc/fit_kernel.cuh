@@ -136,9 +136,12 @@ __device__ __forceinline__ void forward_tiles(const FitView& v, const Layout& L,
 
 // Sub-tiles of at most 16 rows (small minibatches, ragged ends) take 4-row tiles so that all
 // threads share the work; full sub-tiles take 8-row tiles (fewer loads per multiply-add).
+// LEAN kernels (register-capped, see mlp_cv_fit_kernel) always take 4-row tiles: the 8-row tile
+// does not fit beside the gradient tile in their registers.
+template <bool LEAN>
 __device__ __forceinline__ void forward_hidden(const FitView& v, const Layout& L, const float* xs, int d, int dp,
                                                int Hs, int nb, int tid, int nt) {
-  if (nb <= 16) forward_tiles<4>(v, L, xs, d, dp, Hs, nb, tid, nt);
+  if (LEAN || nb <= 16) forward_tiles<4>(v, L, xs, d, dp, Hs, nb, tid, nt);
   else forward_tiles<8>(v, L, xs, d, dp, Hs, nb, tid, nt);
 }
 
@@ -357,7 +360,9 @@ __device__ __forceinline__ void row_delta(const FitView& v, int task, int CS, co
 }
 
 // The whole fit.  CT: class count.  PL: pipelined schedule (extra warps for the output layer).
-template <int CT, int HSC, int DPC, bool PL>
+// LEAN: the kernel is built for fewer registers per thread than its tiles like (smaller forward
+// tile, one operand set in the gradient loop); results are the same bit for bit.
+template <int CT, int HSC, int DPC, bool PL, bool LEAN>
 __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, BlockShared& sh) {
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
   const int2 cf = a.fits[q];
@@ -562,22 +567,31 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
       // gW1 tile: rows k0..k0+7, columns jA..jA+3 and jB..jB+3, b ascending
       auto gw1_phase = [&](const float* xs, const float* A1b, int nb) {
         if (has_tile) {
-          // Two operand sets in flight: the loads of row b + 1 are issued before the multiply-adds
-          // of row b, so a warp does not sit out the shared-memory latency once per row.
           const float* xp = xs + k0;
           const float* da = A1b + jA;
           const float* db = A1b + jB;
-          GradOperands opA, opB;
-          opA.load(xp, da, db, 0, dp, L.WP);
-          int b = 0;
+          if constexpr (LEAN) {
+            GradOperands op;
 #pragma unroll 1
-          for (; b + 2 <= nb; b += 2) {
-            opB.load(xp, da, db, b + 1, dp, L.WP);
-            opA.accumulate(g1);
-            opA.load(xp, da, db, b + 2 < nb ? b + 2 : b, dp, L.WP);
-            opB.accumulate(g1);
+            for (int b = 0; b < nb; ++b) {
+              op.load(xp, da, db, b, dp, L.WP);
+              op.accumulate(g1);
+            }
+          } else {
+            // Two operand sets in flight: the loads of row b + 1 are issued before the multiply-adds
+            // of row b, so a warp does not sit out the shared-memory latency once per row.
+            GradOperands opA, opB;
+            opA.load(xp, da, db, 0, dp, L.WP);
+            int b = 0;
+#pragma unroll 1
+            for (; b + 2 <= nb; b += 2) {
+              opB.load(xp, da, db, b + 1, dp, L.WP);
+              opA.accumulate(g1);
+              opA.load(xp, da, db, b + 2 < nb ? b + 2 : b, dp, L.WP);
+              opB.accumulate(g1);
+            }
+            if (b < nb) opA.accumulate(g1);
           }
-          if (b < nb) opA.accumulate(g1);
         }
       };
       // prefetch of the sub-tile that follows (t0 of step s0) in this epoch into row buffer `into`
@@ -601,7 +615,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           const float* xs = v.Xs + buf * TB * dp;
           const float* ysb = v.ys + buf * TB;
           prefetch_next(t0, buf ^ 1);
-          forward_hidden(v, L, xs, d, dp, Hs, nb, tid, nt);
+          forward_hidden<LEAN>(v, L, xs, d, dp, Hs, nb, tid, nt);
           __syncthreads();
           BBO_PHASE(3);
           output_phase(v.A1, ysb, nb, t0, 0, n_warps);
@@ -636,7 +650,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
             if (tid < nt_main) {
               FitView vv = v;
               vv.A1 = A1cur;
-              forward_hidden(vv, L, v.Xs + xb * TB * dp, d, dp, Hs, nb, tid, nt_main);
+              forward_hidden<LEAN>(vv, L, v.Xs + xb * TB * dp, d, dp, Hs, nb, tid, nt_main);
             }
           }
           __syncthreads();
@@ -686,14 +700,9 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         // Every lane of a tile-owner warp walks the eight tile rows, two at a time (the
         // tensor-memory accesses are warp-wide); lanes without a tile, and rows k >= d, touch only
         // their own moments.  Two rows give sixteen independent update chains, which is what
-        // keeps a lone warp's pipeline busy; the moments of the next pair are requested before
-        // the current pair is updated.
-        uint32_t mr[2][16], vr[2][16];
-        auto request = [&](int pr, int buf) {
-          tmem_load16_issue(tm + 16u * pr, mr[buf]);
-          tmem_load16_issue(tm + 64u + 16u * pr, vr[buf]);
-        };
-        request(0, 0);
+        // keeps a lone warp's pipeline busy.  (Requesting the next pair's moments ahead of the
+        // update cost 32 registers and gained nothing.)
+        uint32_t mr[16], vr[16];
 #pragma unroll
         for (int pr = 0; pr < 4; ++pr) {
           const int i0 = 2 * pr;
@@ -712,13 +721,14 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
               w16[8] = wA.x; w16[9] = wA.y; w16[10] = wA.z; w16[11] = wA.w; w16[12] = wB.x; w16[13] = wB.y; w16[14] = wB.z; w16[15] = wB.w;
             }
           };
+          tmem_load16_issue(tm + 16u * pr, mr);
+          tmem_load16_issue(tm + 64u + 16u * pr, vr);
           load_w();
-          tmem_wait_loads16(mr[pr & 1], vr[pr & 1]);
-          if (pr + 1 < 4) request(pr + 1, (pr + 1) & 1);
+          tmem_wait_loads16(mr, vr);
           float m16[16], v16[16], g16[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            m16[j] = __uint_as_float(mr[pr & 1][j]); v16[j] = __uint_as_float(vr[pr & 1][j]);
+            m16[j] = __uint_as_float(mr[j]); v16[j] = __uint_as_float(vr[j]);
             g16[j] = __fmaf_rn(aB, w16[j], g1[i0 + (j >> 3)][j & 7]);
           }
           if (sgd) {
@@ -801,7 +811,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
     else stage_rows_async(a, a.X, a.y, v, dp, 0, nb, [&](int r) { return a.pi[vb + t0 + r]; }, tid, nt);
     cp_async_wait_all();
     __syncthreads();
-    forward_hidden(v, L, v.Xs, d, dp, Hs, nb, tid, nt);
+    forward_hidden<LEAN>(v, L, v.Xs, d, dp, Hs, nb, tid, nt);
     __syncthreads();
     for (int r0 = warp * 16; r0 < nb; r0 += n_warps * 16) {  // warp-uniform
       const int brow = r0 + (lane >> 1);
@@ -874,11 +884,14 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 }
 
 // One CTA per fit; blockIdx.x indexes this launch's fit list (costliest first).
+// The launch bounds cap the registers at 65,536 / (MINB x NTMAX); a scheduler's quarter of the
+// register file holds two warps at 255 registers, so instances built for more than eight
+// resident warps get about 168 and take the lean forms of the tile loops.
 template <int CT, int HSC, int DPC, int NTMAX, int MINB, bool PL = false>
 __global__ void __launch_bounds__(NTMAX, MINB) mlp_cv_fit_kernel(const FitArgs a) {
   extern __shared__ __align__(16) float smem[];
   __shared__ BlockShared sh;
-  run_fit<CT, HSC, DPC, PL>(a, blockIdx.x, smem, sh);
+  run_fit<CT, HSC, DPC, PL, (MINB * NTMAX > 256)>(a, blockIdx.x, smem, sh);
 }
 
 }  // namespace bbo
