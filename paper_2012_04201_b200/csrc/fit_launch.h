@@ -25,9 +25,9 @@ inline int pipe_extra_warps(int Hs) { return (Hs + 31) / 32 * 32 + 64 <= kMaxFit
 // their registers at 65,536 / (CTAs x threads), and shared memory admits that many (the row
 // buffers and parameters of a fit of that width, moments of W1 in tensor memory).  Four fits per
 // SM up to width 64 and two up to 128 keep about 250 registers per thread.  Widths 136..176 (five
-// or six warps) also run two per SM, at 168 registers and a few hundred bytes of spills: a lone
-// CTA is then 40 % slower, but two of them share an SM at a cost of 10 %, which beats one CTA
-// with the pipelined schedule by 8 %.  Three CTAs of widths 72..96 at 168 registers were 12 %
+// or six warps) also run two per SM, at 168 registers with the lean forms of the tile loops
+// (fit_kernel.cuh) and about two hundred bytes of spills: a lone CTA is then slower, but two of
+// them share an SM at a cost of 10 %, which beats one CTA with the pipelined schedule.  Three CTAs of widths 72..96 at 168 registers were 12 %
 // slower than two at 250.  Widths from 184 sit alone on their SM (shared memory) and take the
 // pipelined schedule.
 constexpr int fast_threads(int Hs) { return (Hs + 31) / 32 * 32; }
