@@ -202,6 +202,32 @@ def test_edge_cases(binding):
     check_against_oracle(gpu, ref, "edge-reg-d7")
 
 
+def test_weights_that_decay_into_denormals_stay_bit_equal(binding):
+    # Two constant-zero feature columns: their weights see only the L2 term, decay geometrically
+    # and end up denormal together with their gradients and first moments, so m / (sqrt(v) + eps)
+    # is denormal for most of the fit.  The update's fast path must give the IEEE quotient there.
+    wl = W.workload("iris8")
+    X = np.concatenate([wl["X"], np.zeros((wl["X"].shape[0], 2), np.float32)], axis=1)
+    cfg = make_configs([
+        (16, 16, 150, 1e-2, 1e-3, 0.9, 0.999, 1e-8),
+        (24, 8, 400, 1e-1, 3e-3, 0.9, 0.999, 1e-8),
+        (40, 16, 400, 1e-1, 1e-2, 0.9, 0.999, 1e-8),
+    ])
+    for task, y in ((0, wl["y"]), (1, wl["X"][:, 0].copy())):   # classification and regression kernels
+        w2 = dict(X=X, y=y, task=task, n_folds=5, seed=5)
+        gpu = gpu_eval(binding, w2, cfg, keep_theta=True)
+        ref = oracle.cv_eval(X, y, task, 5, cfg, 5)
+        exact = check_against_oracle(gpu, ref, f"denormal-task{task}")
+        th = oracle.cv_fits(X, y, task, 5, cfg, 5, [2], [4], want_theta=True)["theta"]
+        w1 = th[: 6 * 40].reshape(6, 40)[4:]                    # weights of the two zero columns
+        tiny = np.abs(w1[w1 != 0.0]) < 1.1754944e-38
+        print(f"[denormal-task{task}] zero-column weights: {tiny.sum()} of {w1.size} denormal, bit-equal parameters:",
+              np.array_equal(gpu["theta"].astype(np.float64), th))
+        assert tiny.sum() + np.sum(w1 == 0.0) >= w1.size // 2      # the regime is actually reached
+        assert np.array_equal(gpu["theta"].astype(np.float64), th)
+        assert exact == 1.0
+
+
 def test_score_depends_only_on_own_config_and_is_deterministic(binding):
     wl = W.workload("breast128", n_configs=12, epochs=8)
     a = gpu_eval(binding, wl, wl["configs"])
