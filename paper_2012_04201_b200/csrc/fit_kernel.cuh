@@ -707,6 +707,12 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         for (int pr = 0; pr < 4; ++pr) {
           const int i0 = 2 * pr;
           const bool live0 = has_tile && (k0 + i0) < d, live1 = has_tile && (k0 + i0 + 1) < d;
+          if constexpr (DPC == 0) {
+            // Feature counts that are not a multiple of eight leave padding rows in the last row
+            // block; where a row pair is padding for every lane of the warp (always so when d < 8)
+            // its moments stay zero and the pair is skipped.
+            if (__all_sync(0xffffffffu, !live0 && !live1)) continue;
+          }
           const int offA = L.oW1 + (k0 + i0) * Hs + jA, offB = L.oW1 + (k0 + i0) * Hs + jB;
           float w16[16];
 #pragma unroll
