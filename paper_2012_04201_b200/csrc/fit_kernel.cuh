@@ -30,6 +30,7 @@
 // access of the hot loops is base + immediate.
 #pragma once
 #include <cstdint>
+#include <type_traits>
 #include <cuda_runtime.h>
 
 #include "device_math.cuh"
@@ -701,17 +702,24 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
         // tensor-memory accesses are warp-wide); lanes without a tile, and rows k >= d, touch only
         // their own moments.  Two rows give sixteen independent update chains, which is what
         // keeps a lone warp's pipeline busy.  (Requesting the next pair's moments ahead of the
-        // update cost 32 registers and gained nothing.)
+        // update cost 32 registers and gained nothing.)  The gradient tile is consumed: it is
+        // zeroed at the start of the next step anyway.
         uint32_t mr[16], vr[16];
+        auto next_rows = [&]() {  // rows 2, 3, .. of the gradient tile move up by two
 #pragma unroll
-        for (int pr = 0; pr < 4; ++pr) {
+          for (int r = 0; r < 6; ++r)
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) g1[r][cc] = g1[r + 2][cc];
+        };
+        auto pair_update = [&](int pr, auto R0) {  // rows 2 pr, 2 pr + 1 of the tile, held in g1[r0], g1[r0 + 1]
+          constexpr int r0 = decltype(R0)::value;
           const int i0 = 2 * pr;
           const bool live0 = has_tile && (k0 + i0) < d, live1 = has_tile && (k0 + i0 + 1) < d;
           if constexpr (DPC == 0) {
             // Feature counts that are not a multiple of eight leave padding rows in the last row
             // block; where a row pair is padding for every lane of the warp (always so when d < 8)
             // its moments stay zero and the pair is skipped.
-            if (__all_sync(0xffffffffu, !live0 && !live1)) continue;
+            if (__all_sync(0xffffffffu, !live0 && !live1)) return;
           }
           const int offA = L.oW1 + (k0 + i0) * Hs + jA, offB = L.oW1 + (k0 + i0) * Hs + jB;
           float w16[16];
@@ -735,7 +743,7 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             m16[j] = __uint_as_float(mr[j]); v16[j] = __uint_as_float(vr[j]);
-            g16[j] = __fmaf_rn(aB, w16[j], g1[i0 + (j >> 3)][j & 7]);
+            g16[j] = __fmaf_rn(aB, w16[j], g1[r0 + (j >> 3)][j & 7]);
           }
           if (sgd) {
             sgd_group<16>(w16, m16, g16, c.lr, beta1);
@@ -754,6 +762,28 @@ __device__ __forceinline__ void run_fit(const FitArgs& a, int q, float* smem, Bl
           }
           tmem_store16(tm + 16u * pr, m16);
           tmem_store16(tm + 64u + 16u * pr, v16);
+        };
+        // The pair loop is rolled, with the tile's rows moved up between iterations (register
+        // arrays cannot be indexed by the loop counter): unrolled it is 35 KB of code that runs
+        // once per step, and CTAs of different widths on one SM, running different instances,
+        // were starving each other of instructions.  Register-capped instances roll two pairs
+        // per iteration (one pair per iteration cost them 5 to 8 %).
+        if constexpr (!LEAN) {
+#pragma unroll 1
+          for (int pr = 0; pr < 4; ++pr) {
+            pair_update(pr, std::integral_constant<int, 0>{});
+            next_rows();
+          }
+        } else {
+#pragma unroll 1
+          for (int hf = 0; hf < 2; ++hf) {
+            pair_update(2 * hf, std::integral_constant<int, 0>{});
+            pair_update(2 * hf + 1, std::integral_constant<int, 2>{});
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+              for (int cc = 0; cc < 8; ++cc) g1[r][cc] = g1[r + 4][cc];
+          }
         }
         tmem_wait_stores();
       }
