@@ -40,12 +40,12 @@ UNIT = "fits/s"
 SM_COUNT_FP32_LANES = 128  # FP32 lanes per SM on sm_100
 # dram__bytes_read.sum + dram__bytes_write.sum of one fit-kernel launch on the digits-shaped data
 # (ncu capture of a 60-fit launch, summarised in profiles/mlp_cv_fit_kernel_small_cases_full.md;
-# a 592-fit launch of the same capture set read 658,176):
+# a 592-fit launch of the same capture set read 627,968):
 # the dataset, the labels, the configurations and the fit list, read once.  It does not grow with
 # the number of fits in the launch, because weights, moments and activations never leave the SM
 # and every later read of X hits the L2; so the figure is not scaled to the bench's launch size.
 # Other workloads have no capture of their own and report null.
-FIT_KERNEL_DRAM_BYTES_PER_LAUNCH = {"digits_sweep": 644352, "digits2048": 644352}
+FIT_KERNEL_DRAM_BYTES_PER_LAUNCH = {"digits_sweep": 615168, "digits2048": 615168}
 
 
 def parse_args():
